@@ -1,0 +1,174 @@
+/*
+ * libtopk — the per-step compression pipeline of bidirectional top_K SGD
+ * (arXiv 2209.15203) on one NVIDIA B200 (sm_100a).
+ *
+ * The N workers of the parameter-server iteration are the N rows of one fp32
+ * tensor on one GPU.  One step (tk_step) does, entirely on the device:
+ *   1. uplink    Top_K_up of every row                (Algorithm 1/2, worker: SEND(Top_K(a^q)))
+ *   2. server    g = sum_{q=1..N} p_q Top_K(a^q), summed in worker order
+ *                                                     (Algorithm 1/2, server step)
+ *   3. downlink  Top_K_down(g) when bidirectional     (Algorithm 2, server: SEND(Top_K(g)));
+ *                g itself when unidirectional         (Algorithm 1, server: SEND(g))
+ *   4. update    w <- w - alpha * message             (Algorithm 1/2, last worker step)
+ * This is the iteration with the error memories epsilon, delta at zero (their
+ * value at t = 1); the step size multiplies the message rather than the
+ * gradient, which selects the same components because Top_K is positively
+ * homogeneous.
+ *
+ * Top_K(x) keeps the K components of largest magnitude (Section 1).  Magnitudes
+ * are compared through the integer key  bits(x) & 0x7fffffff  (so -0 == +0,
+ * denormals are kept, NaN/Inf are ordered by bit pattern); among equal
+ * magnitudes the LOWER index is kept.  A message always has exactly K entries
+ * (zero-valued ones included when the vector has fewer than K non-zeros) and is
+ * listed in ascending index order; values are the original signed values, bit
+ * for bit.  All fp32 arithmetic is round-to-nearest with one rounding per
+ * multiply and one per add/subtract (no fused multiply-add, no flush to zero).
+ *
+ * Conventions
+ *   - "dev" pointers are device memory of the current CUDA device, "host"
+ *     pointers are host memory.  The library never takes ownership of a
+ *     caller's buffer.  fp32 / int32 buffers must be 4-byte aligned; rows of a
+ *     [rows][d] tensor are contiguous (row r starts at element r*d).
+ *   - Every function returns TK_OK (0) or a negative TK_ERR_* code; nothing
+ *     throws or aborts.  tk_strerror() names a code.
+ *   - Work is enqueued on the context's stream and the call returns without
+ *     waiting, except where a function is documented to synchronise.
+ *   - A context may be used by one host thread at a time.
+ */
+#ifndef TOPK_H_
+#define TOPK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tk_ctx tk_ctx;
+
+enum {
+    TK_OK = 0,
+    TK_ERR_INVALID = -1,  /* bad argument (range, NULL, alignment, size) */
+    TK_ERR_ALLOC = -2,    /* workspace too small / allocation failed */
+    TK_ERR_CUDA = -3,     /* a CUDA runtime call failed */
+    TK_ERR_TIMEOUT = -4,  /* a bounded device-side wait expired */
+    TK_ERR_INTERNAL = -5  /* a device-side consistency check failed */
+};
+
+enum {
+    TK_MODE_UNI = 0,   /* Algorithm 1: the downlink carries the aggregate itself */
+    TK_MODE_BIDIR = 1  /* Algorithm 2: the downlink carries Top_K_down of the aggregate */
+};
+
+/* Counters of the last step / selection, filled by tk_status(). */
+typedef struct tk_stats {
+    int32_t device_status;    /* sticky TK_ERR_* raised by a kernel, 0 if none */
+    int32_t rows_general;     /* rows whose predicted threshold failed verification in the
+                                 last selection and were redone by the exact multi-pass path */
+    int64_t union_size;       /* |U|: distinct indices in the last aggregate (<= N*K_up);
+                                 |U|/d is the non-zero fraction of Section 4.2 */
+    int64_t downlink_count;   /* entries applied to w in the last step */
+    int64_t cand_min;         /* fewest / most candidates any row kept in the last uplink */
+    int64_t cand_max;
+    float   select_ms_sum;    /* device time of the streaming selection passes recorded since the
+                                 previous tk_status call, and how many were recorded (both 0 */
+    int32_t select_samples;   /* unless tk_set_profile(ctx, 1); at most 256 are kept) */
+} tk_stats;
+
+/* Bytes of device workspace tk_init needs for these sizes (0 if they are invalid). */
+size_t tk_workspace_bytes(int64_t d, int32_t N, int64_t K_up, int64_t K_down);
+
+/*
+ * Create a context for N workers with vectors of length d (the problem of
+ * Eq. 1: minimise sum_q p_q F^q(w), w in R^d).
+ *   out             receives the context
+ *   d               1 <= d < 2^31
+ *   N               >= 1
+ *   K_up, K_down    1 <= K <= d   (Section 4.2's K_uplink, K_downlink)
+ *   p_host          [N] weights p_q, finite and >= 0 (copied; the sum is not checked)
+ *   workspace_dev   device buffer of at least tk_workspace_bytes() bytes, 256-byte
+ *                   aligned, owned by the caller and kept alive until tk_destroy;
+ *                   the library keeps all per-step state in it and zeroes what
+ *                   it needs here (this call synchronises the stream)
+ *   cuda_stream     a cudaStream_t (NULL = the legacy default stream)
+ */
+int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down,
+            const float* p_host, void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * One iteration (stages 1-4 above).
+ *   w_dev      [d]     parameters, updated in place
+ *   grads_dev  [N][d]  the workers' vectors, read only
+ *   alpha      finite step size
+ *   mode       TK_MODE_UNI or TK_MODE_BIDIR
+ * Asynchronous.  Inputs are assumed finite.
+ */
+int tk_step(tk_ctx* ctx, float* w_dev, const float* grads_dev, float alpha, int mode);
+
+/*
+ * The same iteration for callers whose data lives in host memory: copies
+ * grads_host ([N][d]) and w_host ([d]) to staging buffers the context allocates
+ * on first use (cudaMalloc, 4*(N+1)*d bytes), runs tk_step, copies w back and
+ * synchronises.  Pinned host memory makes the copies fast but is not required.
+ */
+int tk_step_host(tk_ctx* ctx, float* w_host, const float* grads_host, float alpha, int mode);
+
+/*
+ * Top_K of every row of x (stage 1 alone; Section 1's compressor).
+ *   ctx        a context (its stream is used), or NULL for the legacy default stream
+ *   x_dev      [rows][d]
+ *   idx_out_dev, val_out_dev   [rows][K], ascending index per row
+ * rows, d, K need not match the context.  Scratch memory is taken from a
+ * per-process pool that grows with cudaMalloc when a larger problem arrives
+ * (tk_release_scratch frees it).  Asynchronous unless the pool has to grow.
+ */
+int tk_topk(tk_ctx* ctx, const float* x_dev, int32_t rows, int64_t d, int64_t K,
+            int32_t* idx_out_dev, float* val_out_dev);
+
+/* Change K_downlink of an existing context (1 <= K_down <= d). */
+int tk_set_kdown(tk_ctx* ctx, int64_t K_down);
+
+/*
+ * Messages of the last tk_step, for inspection.  Each call synchronises, sorts a
+ * copy by index and writes it to caller-provided device buffers.
+ *   tk_last_uplink     the N uplink messages, [N][K_up]
+ *   tk_last_aggregate  the aggregate g as (index, value) over the union U of the
+ *                      uplink index sets (g is zero elsewhere); buffers of
+ *                      min(N*K_up, d) entries; *count_host = |U|
+ *   tk_last_downlink   the downlink message: Top_K_down(g) with exactly K_down
+ *                      entries (bidirectional; buffers of K_down entries), or g on
+ *                      U (unidirectional; buffers of min(N*K_up, d) entries)
+ */
+int tk_last_uplink(tk_ctx* ctx, int32_t* idx_out_dev, float* val_out_dev);
+int tk_last_aggregate(tk_ctx* ctx, int32_t* idx_out_dev, float* val_out_dev, int64_t* count_host);
+int tk_last_downlink(tk_ctx* ctx, int32_t* idx_out_dev, float* val_out_dev, int64_t* count_host);
+
+/* Synchronise the stream and report counters and the sticky device status. */
+int tk_status(tk_ctx* ctx, tk_stats* out);
+
+/* Record device timestamps around the streaming selection pass of each step (0/1). */
+int tk_set_profile(tk_ctx* ctx, int on);
+
+/*
+ * Testing aid: force every selection of this context down the exact multi-pass
+ * path (1) or back to the predicted single-pass path with verification (0).
+ * Both give identical results.
+ */
+int tk_set_force_general(tk_ctx* ctx, int on);
+
+/* Kernels launched on the context's stream since tk_init. */
+int64_t tk_launch_count(tk_ctx* ctx);
+
+/* Free the host-side context (and its staging buffers).  The workspace stays the caller's. */
+void tk_destroy(tk_ctx* ctx);
+
+/* Free the scratch pool used by tk_topk and the tk_last_* calls. */
+void tk_release_scratch(void);
+
+const char* tk_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOPK_H_ */

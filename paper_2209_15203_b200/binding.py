@@ -1,0 +1,217 @@
+"""ctypes binding of libtopk.so — argument marshalling only.
+
+Every function has the name and the meaning of its C counterpart in
+``include/topk.h``; tensors are passed as raw device pointers.  PyTorch is used
+for device memory and streams, nothing else: all computation happens in the
+library's CUDA kernels.  There is no fallback: if the library is missing or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+from . import build as _build
+
+TK_MODE_UNI = 0
+TK_MODE_BIDIR = 1
+
+EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_set_kdown",
+           "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
+           "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
+
+
+class TkError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed: %s (%d)" % (what, strerror(code), code))
+        self.code = code
+
+
+class tk_stats(ctypes.Structure):
+    _fields_ = [("device_status", ctypes.c_int32), ("rows_general", ctypes.c_int32),
+                ("union_size", ctypes.c_int64), ("downlink_count", ctypes.c_int64),
+                ("cand_min", ctypes.c_int64), ("cand_max", ctypes.c_int64),
+                ("select_ms_sum", ctypes.c_float), ("select_samples", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Open libtopk.so (building it first when the sources are newer and nvcc exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        try:
+            _build.build()
+        except Exception:
+            if not os.path.exists(_build.LIB):
+                raise
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError("libtopk.so is missing; run `python -m paper_2209_15203_b200.build`")
+    lib = ctypes.CDLL(_build.LIB)
+    vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float
+    lib.tk_workspace_bytes.argtypes = [i64, i32, i64, i64]
+    lib.tk_workspace_bytes.restype = ctypes.c_size_t
+    lib.tk_init.argtypes = [ctypes.POINTER(vp), i64, i32, i64, i64, vp, vp, ctypes.c_size_t, vp]
+    lib.tk_step.argtypes = [vp, vp, vp, f32, ctypes.c_int]
+    lib.tk_step_host.argtypes = [vp, vp, vp, f32, ctypes.c_int]
+    lib.tk_topk.argtypes = [vp, vp, i32, i64, i64, vp, vp]
+    lib.tk_set_kdown.argtypes = [vp, i64]
+    lib.tk_last_uplink.argtypes = [vp, vp, vp]
+    lib.tk_last_aggregate.argtypes = [vp, vp, vp, ctypes.POINTER(i64)]
+    lib.tk_last_downlink.argtypes = [vp, vp, vp, ctypes.POINTER(i64)]
+    lib.tk_status.argtypes = [vp, ctypes.POINTER(tk_stats)]
+    lib.tk_set_profile.argtypes = [vp, ctypes.c_int]
+    lib.tk_set_force_general.argtypes = [vp, ctypes.c_int]
+    lib.tk_launch_count.argtypes = [vp]
+    lib.tk_launch_count.restype = i64
+    lib.tk_destroy.argtypes = [vp]
+    lib.tk_destroy.restype = None
+    lib.tk_release_scratch.argtypes = []
+    lib.tk_release_scratch.restype = None
+    lib.tk_strerror.argtypes = [ctypes.c_int]
+    lib.tk_strerror.restype = ctypes.c_char_p
+    for name in ("tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_set_kdown", "tk_last_uplink",
+                 "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile", "tk_set_force_general"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().tk_strerror(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise TkError(code, what)
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype) -> int:
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise ValueError("expected a contiguous CUDA tensor of dtype %s" % dtype)
+    return t.data_ptr()
+
+
+def tk_workspace_bytes(d: int, N: int, K_up: int, K_down: int) -> int:
+    return int(load().tk_workspace_bytes(d, N, K_up, K_down))
+
+
+class Context:
+    """Owns a tk_ctx and the workspace tensor it lives in."""
+
+    def __init__(self, d: int, N: int, K_up: int, K_down: int, p: torch.Tensor,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        lib = load()
+        self.d, self.N, self.K_up, self.K_down = d, N, K_up, K_down
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        nbytes = tk_workspace_bytes(d, N, K_up, K_down)
+        if nbytes == 0:
+            raise TkError(-1, "tk_workspace_bytes")
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            p_host = p.detach().to("cpu", torch.float32).contiguous()
+            handle = ctypes.c_void_p()
+            _check(lib.tk_init(ctypes.byref(handle), d, N, K_up, K_down, p_host.data_ptr(),
+                               self.workspace.data_ptr(), nbytes, self.stream.cuda_stream), "tk_init")
+        self._h = handle
+        self.ucap = min(N * K_up, d)
+        self.last_mode = None
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            load().tk_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the calls of include/topk.h --
+    def tk_step(self, w: torch.Tensor, grads: torch.Tensor, alpha: float, mode: int) -> None:
+        assert w.numel() == self.d and grads.numel() == self.N * self.d
+        _check(load().tk_step(self._h, _dev(w, torch.float32), _dev(grads, torch.float32), alpha, mode), "tk_step")
+        self.last_mode = mode
+
+    def tk_step_host(self, w_host: torch.Tensor, grads_host: torch.Tensor, alpha: float, mode: int) -> None:
+        for t in (w_host, grads_host):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != torch.float32:
+                raise ValueError("expected contiguous float32 host tensors")
+        assert w_host.numel() == self.d and grads_host.numel() == self.N * self.d
+        with torch.cuda.device(self.device):
+            _check(load().tk_step_host(self._h, w_host.data_ptr(), grads_host.data_ptr(), alpha, mode),
+                   "tk_step_host")
+        self.last_mode = mode
+
+    def tk_topk(self, x: torch.Tensor, K: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        return tk_topk(x, K, ctx=self)
+
+    def tk_set_kdown(self, K_down: int) -> None:
+        _check(load().tk_set_kdown(self._h, K_down), "tk_set_kdown")
+        self.K_down = K_down
+
+    def tk_last_uplink(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        idx = torch.empty((self.N, self.K_up), dtype=torch.int32, device=self.device)
+        val = torch.empty((self.N, self.K_up), dtype=torch.float32, device=self.device)
+        _check(load().tk_last_uplink(self._h, idx.data_ptr(), val.data_ptr()), "tk_last_uplink")
+        return idx, val
+
+    def _msg(self, fn, name: str, n: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        idx = torch.empty(n, dtype=torch.int32, device=self.device)
+        val = torch.empty(n, dtype=torch.float32, device=self.device)
+        count = ctypes.c_int64(0)
+        _check(fn(self._h, idx.data_ptr(), val.data_ptr(), ctypes.byref(count)), name)
+        return idx[:count.value], val[:count.value]
+
+    def tk_last_aggregate(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        return self._msg(load().tk_last_aggregate, "tk_last_aggregate", self.ucap)
+
+    def tk_last_downlink(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        n = self.K_down if self.last_mode == TK_MODE_BIDIR else self.ucap
+        return self._msg(load().tk_last_downlink, "tk_last_downlink", max(n, 1))
+
+    def tk_status(self, check: bool = True) -> tk_stats:
+        st = tk_stats()
+        rc = load().tk_status(self._h, ctypes.byref(st))
+        if check:
+            _check(rc, "tk_status")
+        return st
+
+    def tk_set_profile(self, on: bool) -> None:
+        _check(load().tk_set_profile(self._h, 1 if on else 0), "tk_set_profile")
+
+    def tk_set_force_general(self, on: bool) -> None:
+        _check(load().tk_set_force_general(self._h, 1 if on else 0), "tk_set_force_general")
+
+    def tk_launch_count(self) -> int:
+        return int(load().tk_launch_count(self._h))
+
+
+def tk_topk(x: torch.Tensor, K: int, ctx: Optional[Context] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Top_K of every row of x ([rows][d] or [d]): (idx int32, val float32), ascending index."""
+    x2 = x if x.dim() == 2 else x.reshape(1, -1)
+    rows, d = x2.shape
+    idx = torch.empty((rows, K), dtype=torch.int32, device=x.device)
+    val = torch.empty((rows, K), dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(load().tk_topk(ctx._h if ctx is not None else None, _dev(x2, torch.float32), rows, d, K,
+                              idx.data_ptr(), val.data_ptr()), "tk_topk")
+    if x.dim() == 1:
+        return idx[0], val[0]
+    return idx, val
+
+
+def tk_release_scratch() -> None:
+    load().tk_release_scratch()

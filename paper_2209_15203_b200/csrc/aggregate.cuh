@@ -1,0 +1,108 @@
+// Server step of Algorithm 1/2:  g = sum_{q=1..N} p_q Top_K(a^q),  summed in
+// worker order so that the fp32 result does not depend on scheduling.
+//
+// The dense server buffer (one 32-bit word per coordinate, all zero between
+// steps) is the scatter target: agg_link threads every uplink entry onto a
+// per-coordinate chain headed in that buffer; agg_reduce lets the entry at the
+// head of each chain walk it in ascending worker order, accumulate
+//        g_j = fl(g_j + fl(p_q * v_{q,j}))        starting from +0,
+// append (j, g_j) to the union list U, put the word back to zero, and — in
+// unidirectional mode, where the downlink carries g itself — apply
+// w_j <- w_j - alpha g_j  right there (last worker step of Algorithm 1).
+// The work is O(N K_up); no pass over the d coordinates is ever made.
+#pragma once
+
+#include "common.cuh"
+
+namespace tk {
+
+__global__ void __launch_bounds__(256)
+agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, Ctrl* ctrl, u32 d) {
+    u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    u32 j = up[e].x;
+    if (j >= d) { raise_status(ctrl, -5); next[e] = 0; return; }
+    next[e] = atomicExch(&head[j], e + 1);
+}
+
+__global__ void __launch_bounds__(256)
+agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
+                  u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
+                  uint2* U, u32 ucap, float* w, float alpha, int apply, Ctrl* ctrl, u32 d) {
+    u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+    bool owner = false;
+    u32 j = 0;
+    float acc = 0.0f;
+    if (e < total) {
+        j = up[e].x;
+        owner = j < d && __ldcg(&head[j]) == e + 1;
+    }
+    if (owner) {
+        // walk the chain once per term, each time taking the smallest worker not yet added
+        int last_q = -1;
+        for (u32 guard = 0; guard <= total; ++guard) {
+            int best_q = 0x7fffffff;
+            u32 best_e = 0;
+            for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) {
+                int q = (int)((c - 1) / K_up);
+                if (q > last_q && q < best_q) { best_q = q; best_e = c - 1; }
+            }
+            if (best_q == 0x7fffffff) break;
+            float term = __fmul_rn(p[best_q], __uint_as_float(up[best_e].y));
+            acc = __fadd_rn(acc, term);
+            last_q = best_q;
+        }
+        head[j] = 0;
+        if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
+    }
+    u32 bits = __float_as_uint(acc);
+    u32 m = warp_append(owner, j, bits, &uni->cand_count, U, ucap);
+    if (m) {
+        u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
+        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&uni->max_key, wm);
+    }
+}
+
+// Start-of-step reset of the union's state and the downlink counter.
+__global__ void reset_union_kernel(RowState* uni) {
+    uni->lo = 0;
+    uni->cand_count = 0;
+    uni->max_key = 0;
+    uni->out_count = 0;
+    uni->flags = 0;
+}
+
+// ---- helpers of the inspection calls (not on the per-step path) ----
+
+// Entries of `sel` with a non-zero magnitude go to msg; flags[idx] = 1 marks the ones below `limit`.
+__global__ void msg_collect_kernel(const uint2* sel, u32 n, uint2* msg, u32* msg_count,
+                                   unsigned char* flags, u32 limit) {
+    u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+    bool pred = false;
+    uint2 e = make_uint2(0, 0);
+    if (i < n) {
+        e = sel[i];
+        pred = key_of(e.y) != 0;
+        if (pred && e.x < limit) flags[e.x] = 1;
+    }
+    warp_append(pred, e.x, e.y, msg_count, msg, 0xffffffffu);
+}
+
+// Append the first `pad` indices j in [0, limit) with flags[j] == 0 as (j, +0.0).  One CTA.
+__global__ void __launch_bounds__(1024)
+msg_pad_kernel(const unsigned char* flags, u32 limit, u32 pad, uint2* msg, u32 at) {
+    __shared__ u32 scratch[33];
+    u32 done = 0;
+    for (u32 base = 0; base < limit && done < pad; base += blockDim.x) {
+        u32 j = base + threadIdx.x;
+        u32 free_ = (j < limit && flags[j] == 0) ? 1u : 0u;
+        u32 total;
+        u32 incl = block_inclusive_scan(free_, scratch, &total);
+        u32 rank = done + incl - free_;
+        if (free_ && rank < pad) msg[at + rank] = make_uint2(j, 0u);
+        done += total;
+        __syncthreads();
+    }
+}
+
+}  // namespace tk

@@ -1,0 +1,673 @@
+// Host side of libtopk: argument checking, workspace layout, launch sequences.
+// The C ABI is declared and documented in include/topk.h.
+#include "../../include/topk.h"
+
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+#include <new>
+
+#include "aggregate.cuh"
+#include "common.cuh"
+#include "select.cuh"
+#include "sort.cuh"
+
+using namespace tk;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxEvents = 256;
+
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct DeviceInfo {
+    bool ready = false;
+    int sms = 0;
+    int general_grid = 0;  // co-resident CTAs of general_kernel
+};
+DeviceInfo g_dev[64];
+
+int device_info(DeviceInfo** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
+    DeviceInfo& di = g_dev[dev];
+    if (!di.ready) {
+        int coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TK_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return TK_ERR_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, general_kernel, kStreamThreads, 0) != cudaSuccess ||
+            per_sm < 1)
+            return TK_ERR_CUDA;
+        di.general_grid = per_sm * di.sms;
+        di.ready = true;
+    }
+    *out = &di;
+    return TK_OK;
+}
+
+// ---- buffers of one batched selection -------------------------------------------------------
+struct SelectBufs {
+    RowState* rs = nullptr;   // [rows]
+    u32* hist = nullptr;      // [rows][kHistBins], zero at rest
+    u32* smax = nullptr;      // [rows][kSampleSlots]
+    uint2* cand = nullptr;    // [rows][cap]
+    uint2* out = nullptr;     // [rows][K]
+    u32 cap = 0;
+    u32 tpr = 0;              // tiles per row
+};
+
+struct SelectLayout {
+    size_t off_rs, off_hist, off_smax, off_cand, off_out, bytes;
+    u32 cap, tpr;
+};
+
+u32 candidate_capacity(int64_t d, int64_t K) {
+    int64_t cap = 4 * K + 8192;
+    if (cap > d) cap = d;
+    return (u32)cap;
+}
+
+SelectLayout select_layout(int64_t rows, int64_t d, int64_t K) {
+    SelectLayout L;
+    L.cap = candidate_capacity(d, K);
+    int64_t nv = (d + 3) / 4;
+    int64_t tpr = (nv + kTileVecs - 1) / kTileVecs;
+    L.tpr = (u32)(tpr < 1 ? 1 : tpr);
+    size_t o = 0;
+    L.off_rs = o;   o += align_up((size_t)rows * sizeof(RowState));
+    L.off_hist = o; o += align_up((size_t)rows * kHistBins * sizeof(u32));
+    L.off_smax = o; o += align_up((size_t)rows * kSampleSlots * sizeof(u32));
+    L.off_cand = o; o += align_up((size_t)rows * L.cap * sizeof(uint2));
+    L.off_out = o;  o += align_up((size_t)rows * (size_t)K * sizeof(uint2));
+    L.bytes = o;
+    return L;
+}
+
+SelectBufs bind(const SelectLayout& L, char* base) {
+    SelectBufs b;
+    b.rs = (RowState*)(base + L.off_rs);
+    b.hist = (u32*)(base + L.off_hist);
+    b.smax = (u32*)(base + L.off_smax);
+    b.cand = (uint2*)(base + L.off_cand);
+    b.out = (uint2*)(base + L.off_out);
+    b.cap = L.cap;
+    b.tpr = L.tpr;
+    return b;
+}
+
+// ---- sort scratch ---------------------------------------------------------------------------
+struct SortLayout {
+    size_t off_tmp, off_cnt, bytes;
+    u32 tiles;
+};
+
+SortLayout sort_layout(int64_t rows, int64_t n) {
+    SortLayout L;
+    L.tiles = (u32)((n + kSortTile - 1) / kSortTile);
+    if (L.tiles < 1) L.tiles = 1;
+    size_t o = 0;
+    L.off_tmp = o; o += align_up((size_t)rows * (size_t)n * sizeof(uint2));
+    L.off_cnt = o; o += align_up((size_t)rows * 256 * L.tiles * sizeof(u32));
+    L.bytes = o;
+    return L;
+}
+
+// ---- per-device scratch pool (tk_topk and the inspection calls) ------------------------------
+struct Pool {
+    char* base = nullptr;
+    size_t bytes = 0;
+};
+Pool g_pool[64];
+
+int pool_get(size_t bytes, char** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
+    Pool& p = g_pool[dev];
+    if (p.bytes < bytes) {
+        if (p.base) {
+            if (cudaDeviceSynchronize() != cudaSuccess) return TK_ERR_CUDA;
+            cudaFree(p.base);
+            p.base = nullptr;
+            p.bytes = 0;
+        }
+        size_t want = bytes + bytes / 8;
+        if (cudaMalloc((void**)&p.base, want) != cudaSuccess) {
+            cudaGetLastError();
+            p.base = nullptr;
+            return TK_ERR_ALLOC;
+        }
+        p.bytes = want;
+    }
+    *out = p.base;
+    return TK_OK;
+}
+
+bool aligned4(const void* p) { return p != nullptr && ((uintptr_t)p & 3u) == 0; }
+
+int bits_of(int64_t v) {  // number of significant bits of v >= 0
+    int b = 0;
+    while (v > 0) { ++b; v >>= 1; }
+    return b;
+}
+
+}  // namespace
+
+// ---- the context ------------------------------------------------------------------------------
+struct tk_ctx {
+    int64_t d = 0, K_up = 0, K_down = 0;
+    int32_t N = 0;
+    cudaStream_t stream = nullptr;
+    char* ws = nullptr;
+    size_t ws_bytes = 0;
+    // workspace views
+    Ctrl* ctrl = nullptr;
+    float* p = nullptr;
+    SelectBufs up;             // uplink selection; up.out = the N uplink messages
+    RowState* uni = nullptr;   // state of the union list / downlink selection
+    u32* head = nullptr;       // [d] dense server buffer, zero at rest
+    u32* next = nullptr;       // [N*K_up]
+    uint2* U = nullptr;        // [ucap] aggregate over the union
+    uint2* sel = nullptr;      // [ucap] downlink message (unordered)
+    u32 ucap = 0;
+    // host state
+    int force_general = 0;
+    int profile = 0;
+    int last_mode = -1;
+    int64_t last_kdown = 0;
+    int64_t launches = 0;
+    cudaEvent_t ev[2 * kMaxEvents] = {};
+    bool ev_ready = false;
+    int ev_used = 0;
+    float* stage_g = nullptr;  // tk_step_host staging
+    float* stage_w = nullptr;
+};
+
+namespace {
+
+struct CtxLayout {
+    size_t off_ctrl, off_p, off_sel_up, off_uni, off_head, off_next, off_U, off_sel, bytes;
+    SelectLayout up;
+    u32 ucap;
+};
+
+bool sizes_ok(int64_t d, int64_t N, int64_t K_up, int64_t K_down) {
+    return d >= 1 && d < ((int64_t)1 << 31) && N >= 1 && N <= 65535 && K_up >= 1 && K_up <= d &&
+           K_down >= 1 && K_down <= d && N * K_up < ((int64_t)1 << 31);
+}
+
+CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
+    CtxLayout L;
+    L.up = select_layout(N, d, K_up);
+    int64_t ucap = N * K_up < d ? N * K_up : d;
+    L.ucap = (u32)ucap;
+    size_t o = 0;
+    L.off_ctrl = o;   o += align_up(sizeof(Ctrl));
+    L.off_p = o;      o += align_up((size_t)N * sizeof(float));
+    L.off_sel_up = o; o += L.up.bytes;
+    L.off_uni = o;    o += align_up(sizeof(RowState));
+    L.off_head = o;   o += align_up((size_t)d * sizeof(u32));
+    L.off_next = o;   o += align_up((size_t)(N * K_up) * sizeof(u32));
+    L.off_U = o;      o += align_up((size_t)ucap * sizeof(uint2));
+    L.off_sel = o;    o += align_up((size_t)ucap * sizeof(uint2));
+    L.bytes = o;
+    return L;
+}
+
+int cluster_size_for(int64_t entries) {
+    int64_t want = (entries + 8191) / 8192;
+    int cs = 1;
+    while (cs < 8 && cs < want) cs *= 2;
+    return cs;
+}
+
+#define TK_LAUNCH_CHECK()                                   \
+    do {                                                    \
+        if (cudaGetLastError() != cudaSuccess) return TK_ERR_CUDA; \
+    } while (0)
+
+int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, size_t list_stride, u32 cap,
+                  RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, Ctrl* ctrl) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(rows * cs), 1, 1);
+    cfg.blockDim = dim3(kSelectThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, select_kernel, lists, list_stride, cap, rs, K, out, out_stride, apply, ctrl) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return TK_OK;
+}
+
+// Exact Top_K of every row of x into b.out ([rows][K], arbitrary order).  ev0/ev1, when
+// given, bracket the streaming pass.  *launches is advanced by the kernels enqueued.
+int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
+               Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches) {
+    DeviceInfo* di = nullptr;
+    int rc = device_info(&di);
+    if (rc != TK_OK) return rc;
+    const bool predict = !force_general && d >= 262144 && K * 64 <= d;
+    int spt = 1;
+    u32 groups = 0, rank = 0;
+    if (predict) {
+        int64_t want = (d + 1024 * K - 1) / (1024 * K);
+        int64_t lim = d / 262144 < 16 ? d / 262144 : 16;
+        spt = (int)(want < 1 ? 1 : (want > lim ? lim : want));
+        groups = (u32)kSampleSlots * (u32)spt;
+        double ks = (double)K * 8.0 * groups / (double)d;  // expected top-K members in the sample
+        double r = ceil(ks + 6.0 * sqrt(ks) + 4.0);
+        rank = (u32)(r > kSampleSlots / 2 ? kSampleSlots / 2 : r);
+    }
+    for (int64_t r0 = 0; r0 < rows; r0 += kMaxRowsPerLaunch) {
+        int nr = (int)(rows - r0 < kMaxRowsPerLaunch ? rows - r0 : kMaxRowsPerLaunch);
+        const float* xb = x + (size_t)r0 * (size_t)d;
+        RowState* rs = b.rs + r0;
+        u32* hist = b.hist + (size_t)r0 * kHistBins;
+        u32* smax = b.smax + (size_t)r0 * kSampleSlots;
+        uint2* cand = b.cand + (size_t)r0 * b.cap;
+        uint2* out = b.out + (size_t)r0 * (size_t)K;
+        if (predict) {
+            predict_kernel<<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, spt, groups, rank, rs, smax);
+            TK_LAUNCH_CHECK();
+            if (ev0) cudaEventRecord(ev0, stream);
+            u64 tiles = (u64)nr * b.tpr;
+            u32 grid = (u32)(tiles < (u64)(di->sms * 4) ? tiles : (u64)(di->sms * 4));
+            filter_kernel<<<grid, kStreamThreads, 0, stream>>>(xb, nr, d, b.tpr, rs, cand, b.cap);
+            TK_LAUNCH_CHECK();
+            if (ev1) cudaEventRecord(ev1, stream);
+            *launches += 2;
+        } else {
+            reset_rows_kernel<<<(nr + 255) / 256, 256, 0, stream>>>(rs, nr);
+            TK_LAUNCH_CHECK();
+            *launches += 1;
+        }
+        {
+            u32 Ku = (u32)K, tpr = b.tpr, cap = b.cap;
+            void* args[] = {(void*)&xb, (void*)&nr, (void*)&d, (void*)&Ku, (void*)&tpr, (void*)&cap,
+                            (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl};
+            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kStreamThreads), args,
+                                            0, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return TK_ERR_CUDA;
+            }
+            *launches += 1;
+        }
+        ApplyArgs none = {nullptr, 0.0f};
+        int64_t expect = predict ? 3 * K : (int64_t)b.cap;
+        rc = launch_select(stream, nr, cluster_size_for(expect), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, none,
+                           ctrl);
+        if (rc != TK_OK) return rc;
+        *launches += 1;
+    }
+    return TK_OK;
+}
+
+// Sort `rows` segments of (index, value) entries by index into idx_out / val_out.
+// Segment r starts at src + r*stride and has min(n_fixed, counts[r*count_stride]) entries
+// (n_fixed when counts is NULL).  tmp / cnt come from sort_layout(rows, n_fixed).
+int run_sort(cudaStream_t stream, uint2* src, size_t stride, const u32* counts, size_t count_stride, u32 n_fixed,
+             int64_t rows, int64_t d, uint2* tmp, u32* cnt, u32 tiles, int32_t* idx_out, float* val_out,
+             size_t out_stride, int64_t* launches) {
+    if (n_fixed == 0 || rows == 0) return TK_OK;
+    int passes = (bits_of(d - 1) + 7) / 8;
+    if (passes < 1) passes = 1;
+    uint2* a = src;
+    uint2* bbuf = tmp;
+    for (int64_t r0 = 0; r0 < rows; r0 += 32768) {
+        int nr = (int)(rows - r0 < 32768 ? rows - r0 : 32768);
+        uint2* cur = a + (size_t)r0 * stride;
+        uint2* oth = bbuf + (size_t)r0 * stride;
+        const u32* cn = counts ? counts + (size_t)r0 * count_stride : nullptr;
+        u32* c = cnt + (size_t)r0 * 256 * tiles;
+        for (int p = 0; p < passes; ++p) {
+            int shift = 8 * p;
+            bool final_pass = p == passes - 1;
+            sort_local_kernel<<<dim3(tiles, nr), kSortTile, 0, stream>>>(cur, stride, cn, count_stride, n_fixed, shift,
+                                                                        tiles, c);
+            TK_LAUNCH_CHECK();
+            sort_scan_kernel<<<nr, 256, 0, stream>>>(c, tiles);
+            TK_LAUNCH_CHECK();
+            sort_scatter_kernel<<<dim3(tiles, nr), kSortTile, 0, stream>>>(
+                cur, stride, cn, count_stride, n_fixed, shift, tiles, c, final_pass ? nullptr : oth,
+                idx_out + (size_t)r0 * out_stride, val_out + (size_t)r0 * out_stride, out_stride);
+            TK_LAUNCH_CHECK();
+            *launches += 3;
+            uint2* t = cur; cur = oth; oth = t;
+        }
+    }
+    return TK_OK;
+}
+
+}  // namespace
+
+// ---- C ABI --------------------------------------------------------------------------------------
+extern "C" {
+
+size_t tk_workspace_bytes(int64_t d, int32_t N, int64_t K_up, int64_t K_down) {
+    if (!sizes_ok(d, N, K_up, K_down)) return 0;
+    return ctx_layout(d, N, K_up).bytes;
+}
+
+int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, const float* p_host,
+            void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    if (!out) return TK_ERR_INVALID;
+    *out = nullptr;
+    if (!sizes_ok(d, N, K_up, K_down) || !p_host || !workspace_dev) return TK_ERR_INVALID;
+    if (((uintptr_t)workspace_dev & (kAlign - 1)) != 0) return TK_ERR_INVALID;
+    for (int q = 0; q < N; ++q)
+        if (!isfinite(p_host[q]) || p_host[q] < 0.0f) return TK_ERR_INVALID;
+    CtxLayout L = ctx_layout(d, N, K_up);
+    if (workspace_bytes < L.bytes) return TK_ERR_ALLOC;
+    DeviceInfo* di = nullptr;
+    int rc = device_info(&di);
+    if (rc != TK_OK) return rc;
+    tk_ctx* c = new (std::nothrow) tk_ctx();
+    if (!c) return TK_ERR_ALLOC;
+    c->d = d; c->N = N; c->K_up = K_up; c->K_down = K_down;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->ws = (char*)workspace_dev;
+    c->ws_bytes = workspace_bytes;
+    c->ctrl = (Ctrl*)(c->ws + L.off_ctrl);
+    c->p = (float*)(c->ws + L.off_p);
+    c->up = bind(L.up, c->ws + L.off_sel_up);
+    c->uni = (RowState*)(c->ws + L.off_uni);
+    c->head = (u32*)(c->ws + L.off_head);
+    c->next = (u32*)(c->ws + L.off_next);
+    c->U = (uint2*)(c->ws + L.off_U);
+    c->sel = (uint2*)(c->ws + L.off_sel);
+    c->ucap = L.ucap;
+    // state that must be zero at rest: control block, row states, histograms, the dense buffer
+    bool ok = cudaMemsetAsync(c->ctrl, 0, sizeof(Ctrl), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->up.rs, 0, (size_t)N * sizeof(RowState), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->up.hist, 0, (size_t)N * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->uni, 0, sizeof(RowState), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->head, 0, (size_t)d * sizeof(u32), c->stream) == cudaSuccess &&
+              cudaMemcpyAsync(c->p, p_host, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream) ==
+                  cudaSuccess &&
+              cudaStreamSynchronize(c->stream) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        delete c;
+        return TK_ERR_CUDA;
+    }
+    *out = c;
+    return TK_OK;
+}
+
+int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
+    if (!c || !aligned4(w_dev) || !aligned4(grads_dev) || !isfinite(alpha)) return TK_ERR_INVALID;
+    if (mode != TK_MODE_UNI && mode != TK_MODE_BIDIR) return TK_ERR_INVALID;
+    cudaStream_t s = c->stream;
+    reset_union_kernel<<<1, 1, 0, s>>>(c->uni);
+    TK_LAUNCH_CHECK();
+    c->launches += 1;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
+        e0 = c->ev[2 * c->ev_used];
+        e1 = c->ev[2 * c->ev_used + 1];
+        c->ev_used += 1;
+    }
+    int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
+                        &c->launches);
+    if (rc != TK_OK) return rc;
+    u32 total = (u32)(c->N * c->K_up);
+    u32 blocks = (total + 255) / 256;
+    agg_link_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, c->head, c->next, c->ctrl, (u32)c->d);
+    TK_LAUNCH_CHECK();
+    agg_reduce_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->uni, c->U,
+                                             c->ucap, w_dev, alpha, mode == TK_MODE_UNI ? 1 : 0, c->ctrl, (u32)c->d);
+    TK_LAUNCH_CHECK();
+    c->launches += 2;
+    if (mode == TK_MODE_BIDIR) {
+        ApplyArgs ap = {w_dev, alpha};
+        rc = launch_select(s, 1, 8, c->U, c->ucap, c->ucap, c->uni, (u32)c->K_down, c->sel, c->ucap, ap, c->ctrl);
+        if (rc != TK_OK) return rc;
+        c->launches += 1;
+    }
+    c->last_mode = mode;
+    c->last_kdown = c->K_down;
+    return TK_OK;
+}
+
+int tk_step_host(tk_ctx* c, float* w_host, const float* grads_host, float alpha, int mode) {
+    if (!c || !w_host || !grads_host) return TK_ERR_INVALID;
+    size_t gbytes = (size_t)c->N * (size_t)c->d * sizeof(float), wbytes = (size_t)c->d * sizeof(float);
+    if (!c->stage_g) {
+        if (cudaMalloc((void**)&c->stage_g, gbytes) != cudaSuccess ||
+            cudaMalloc((void**)&c->stage_w, wbytes) != cudaSuccess) {
+            cudaGetLastError();
+            if (c->stage_g) cudaFree(c->stage_g);
+            c->stage_g = nullptr;
+            c->stage_w = nullptr;
+            return TK_ERR_ALLOC;
+        }
+    }
+    if (cudaMemcpyAsync(c->stage_g, grads_host, gbytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaMemcpyAsync(c->stage_w, w_host, wbytes, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+        return TK_ERR_CUDA;
+    int rc = tk_step(c, c->stage_w, c->stage_g, alpha, mode);
+    if (rc != TK_OK) return rc;
+    if (cudaMemcpyAsync(w_host, c->stage_w, wbytes, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return TK_ERR_CUDA;
+    return TK_OK;
+}
+
+int tk_topk(tk_ctx* c, const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
+            float* val_out_dev) {
+    if (!aligned4(x_dev) || !aligned4(idx_out_dev) || !aligned4(val_out_dev)) return TK_ERR_INVALID;
+    if (rows < 1 || d < 1 || d >= ((int64_t)1 << 31) || K < 1 || K > d) return TK_ERR_INVALID;
+    cudaStream_t s = c ? c->stream : nullptr;
+    SelectLayout SL = select_layout(rows, d, K);
+    SortLayout QL = sort_layout(rows, K);
+    size_t off_ctrl = SL.bytes + QL.bytes;
+    char* base = nullptr;
+    int rc = pool_get(off_ctrl + align_up(sizeof(Ctrl)), &base);
+    if (rc != TK_OK) return rc;
+    SelectBufs b = bind(SL, base);
+    Ctrl* ctrl = c ? c->ctrl : (Ctrl*)(base + off_ctrl);
+    if (cudaMemsetAsync(b.rs, 0, (size_t)rows * sizeof(RowState), s) != cudaSuccess ||
+        cudaMemsetAsync(b.hist, 0, (size_t)rows * kHistBins * sizeof(u32), s) != cudaSuccess ||
+        (!c && cudaMemsetAsync(ctrl, 0, sizeof(Ctrl), s) != cudaSuccess))
+        return TK_ERR_CUDA;
+    int64_t local = 0;
+    int64_t* launches = c ? &c->launches : &local;
+    rc = run_select(s, x_dev, rows, d, K, b, ctrl, c ? c->force_general != 0 : false, nullptr, nullptr, launches);
+    if (rc != TK_OK) return rc;
+    return run_sort(s, b.out, (size_t)K, nullptr, 0, (u32)K, rows, d, (uint2*)(base + SL.bytes + QL.off_tmp),
+                    (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, launches);
+}
+
+int tk_set_kdown(tk_ctx* c, int64_t K_down) {
+    if (!c || K_down < 1 || K_down > c->d) return TK_ERR_INVALID;
+    c->K_down = K_down;
+    return TK_OK;
+}
+
+int tk_last_uplink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev) {
+    if (!c || !aligned4(idx_out_dev) || !aligned4(val_out_dev) || c->last_mode < 0) return TK_ERR_INVALID;
+    SortLayout QL = sort_layout(c->N, c->K_up);
+    char* base = nullptr;
+    int rc = pool_get(QL.bytes, &base);
+    if (rc != TK_OK) return rc;
+    rc = run_sort(c->stream, c->up.out, (size_t)c->K_up, nullptr, 0, (u32)c->K_up, c->N, c->d,
+                  (uint2*)(base + QL.off_tmp), (u32*)(base + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev,
+                  (size_t)c->K_up, &c->launches);
+    if (rc != TK_OK) return rc;
+    return cudaStreamSynchronize(c->stream) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+int tk_last_aggregate(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64_t* count_host) {
+    if (!c || !aligned4(idx_out_dev) || !aligned4(val_out_dev) || !count_host || c->last_mode < 0)
+        return TK_ERR_INVALID;
+    RowState u;
+    if (cudaMemcpyAsync(&u, c->uni, sizeof u, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return TK_ERR_CUDA;
+    u32 n = u.cand_count < c->ucap ? u.cand_count : c->ucap;
+    *count_host = n;
+    if (n == 0) return TK_OK;
+    SortLayout QL = sort_layout(1, n);
+    char* base = nullptr;
+    int rc = pool_get(QL.bytes, &base);
+    if (rc != TK_OK) return rc;
+    rc = run_sort(c->stream, c->U, c->ucap, nullptr, 0, n, 1, c->d, (uint2*)(base + QL.off_tmp),
+                  (u32*)(base + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, n, &c->launches);
+    if (rc != TK_OK) return rc;
+    return cudaStreamSynchronize(c->stream) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+int tk_last_downlink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64_t* count_host) {
+    if (!c || c->last_mode < 0) return TK_ERR_INVALID;
+    if (c->last_mode == TK_MODE_UNI) return tk_last_aggregate(c, idx_out_dev, val_out_dev, count_host);
+    if (!aligned4(idx_out_dev) || !aligned4(val_out_dev) || !count_host) return TK_ERR_INVALID;
+    // The step selects among the union only.  The message proper has exactly K_down entries:
+    // every selected entry of non-zero magnitude, then zero-valued entries at the lowest
+    // indices that carry no such entry.
+    RowState u;
+    if (cudaMemcpyAsync(&u, c->uni, sizeof u, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return TK_ERR_CUDA;
+    u32 nsel = u.out_count < c->ucap ? u.out_count : c->ucap;
+    u32 Kd = (u32)c->last_kdown;
+    SortLayout QL = sort_layout(1, Kd);
+    size_t off_msg = QL.bytes;
+    size_t off_flags = off_msg + align_up((size_t)Kd * sizeof(uint2));
+    size_t off_cnt = off_flags + align_up((size_t)Kd);
+    char* base = nullptr;
+    int rc = pool_get(off_cnt + kAlign, &base);
+    if (rc != TK_OK) return rc;
+    uint2* msg = (uint2*)(base + off_msg);
+    unsigned char* flags = (unsigned char*)(base + off_flags);
+    u32* msg_count = (u32*)(base + off_cnt);
+    cudaStream_t s = c->stream;
+    if (cudaMemsetAsync(flags, 0, Kd, s) != cudaSuccess || cudaMemsetAsync(msg_count, 0, sizeof(u32), s) != cudaSuccess)
+        return TK_ERR_CUDA;
+    u32 nz = 0;
+    if (nsel) {
+        msg_collect_kernel<<<(nsel + 255) / 256, 256, 0, s>>>(c->sel, nsel, msg, msg_count, flags, Kd);
+        TK_LAUNCH_CHECK();
+        c->launches += 1;
+    }
+    if (cudaMemcpyAsync(&nz, msg_count, sizeof nz, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return TK_ERR_CUDA;
+    if (nz > Kd) return TK_ERR_INTERNAL;
+    if (nz < Kd) {
+        msg_pad_kernel<<<1, 1024, 0, s>>>(flags, Kd, Kd - nz, msg, nz);
+        TK_LAUNCH_CHECK();
+        c->launches += 1;
+    }
+    *count_host = Kd;
+    rc = run_sort(s, msg, Kd, nullptr, 0, Kd, 1, c->d, (uint2*)(base + QL.off_tmp), (u32*)(base + QL.off_cnt),
+                  QL.tiles, idx_out_dev, val_out_dev, Kd, &c->launches);
+    if (rc != TK_OK) return rc;
+    return cudaStreamSynchronize(s) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+int tk_status(tk_ctx* c, tk_stats* out) {
+    if (!c || !out) return TK_ERR_INVALID;
+    memset(out, 0, sizeof *out);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    Ctrl ctrl;
+    RowState u;
+    RowState* rows = new (std::nothrow) RowState[c->N];
+    if (!rows) return TK_ERR_ALLOC;
+    bool ok = cudaMemcpy(&ctrl, c->ctrl, sizeof ctrl, cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemcpy(&u, c->uni, sizeof u, cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemcpy(rows, c->up.rs, (size_t)c->N * sizeof(RowState), cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (!ok) {
+        delete[] rows;
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    out->device_status = ctrl.status;
+    out->rows_general = (int32_t)ctrl.rows_general;
+    out->union_size = u.cand_count;
+    out->downlink_count = c->last_mode == TK_MODE_BIDIR ? u.out_count : u.cand_count;
+    int64_t lo = INT64_MAX, hi = 0;
+    for (int q = 0; q < c->N; ++q) {
+        int64_t v = rows[q].cand_count;
+        if (v < lo) lo = v;
+        if (v > hi) hi = v;
+    }
+    out->cand_min = lo;
+    out->cand_max = hi;
+    delete[] rows;
+    float sum = 0.0f;
+    for (int i = 0; i < c->ev_used; ++i) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]) == cudaSuccess) sum += ms;
+        else cudaGetLastError();
+    }
+    out->select_ms_sum = sum;
+    out->select_samples = c->ev_used;
+    c->ev_used = 0;
+    return ctrl.status == 0 ? TK_OK : ctrl.status;
+}
+
+int tk_set_profile(tk_ctx* c, int on) {
+    if (!c) return TK_ERR_INVALID;
+    if (on && !c->ev_ready) {
+        for (int i = 0; i < 2 * kMaxEvents; ++i)
+            if (cudaEventCreate(&c->ev[i]) != cudaSuccess) return TK_ERR_CUDA;
+        c->ev_ready = true;
+    }
+    c->profile = on ? 1 : 0;
+    c->ev_used = 0;
+    return TK_OK;
+}
+
+int tk_set_force_general(tk_ctx* c, int on) {
+    if (!c) return TK_ERR_INVALID;
+    c->force_general = on ? 1 : 0;
+    return TK_OK;
+}
+
+int64_t tk_launch_count(tk_ctx* c) { return c ? c->launches : 0; }
+
+void tk_destroy(tk_ctx* c) {
+    if (!c) return;
+    if (c->ev_ready)
+        for (int i = 0; i < 2 * kMaxEvents; ++i) cudaEventDestroy(c->ev[i]);
+    if (c->stage_g) cudaFree(c->stage_g);
+    if (c->stage_w) cudaFree(c->stage_w);
+    delete c;
+}
+
+void tk_release_scratch(void) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    if (g_pool[dev].base) {
+        cudaDeviceSynchronize();
+        cudaFree(g_pool[dev].base);
+        g_pool[dev].base = nullptr;
+        g_pool[dev].bytes = 0;
+    }
+}
+
+const char* tk_strerror(int code) {
+    switch (code) {
+        case TK_OK: return "ok";
+        case TK_ERR_INVALID: return "invalid argument";
+        case TK_ERR_ALLOC: return "workspace too small or allocation failed";
+        case TK_ERR_CUDA: return "CUDA runtime error";
+        case TK_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case TK_ERR_INTERNAL: return "device-side consistency check failed";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

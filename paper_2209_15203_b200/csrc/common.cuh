@@ -1,0 +1,163 @@
+// Shared device-side definitions of libtopk: per-row selection state, the
+// composite ordering key, warp/block primitives.
+//
+// Ordering.  Top_K keeps the K components of largest magnitude (Section 1 of
+// the paper); the library orders components by the pair (key descending, index
+// ascending) with key = bits & 0x7fffffff.  Both are packed into one 64-bit
+// "composite key"
+//        ck = key << 32 | (0xffffffff - index)
+// so that "larger ck" means "kept first" and no two components of a row
+// compare equal.  Top_K is then: the K largest composite keys.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cooperative_groups.h>
+#include <stdint.h>
+
+namespace tk {
+
+namespace cg = cooperative_groups;
+
+typedef unsigned int u32;
+typedef unsigned long long u64;
+
+constexpr int kHistBins = 2048;        // buckets of one refinement level
+constexpr int kPredictCtas = 8;        // sampling CTAs per row
+constexpr int kPredictThreads = 512;
+constexpr int kSampleSlots = kPredictCtas * kPredictThreads;  // per-row sample maxima
+constexpr int kStreamThreads = 512;    // streaming kernels: threads per CTA
+constexpr int kStreamUnroll = 4;       // 16-byte loads in flight per thread
+constexpr int kTileVecs = kStreamThreads * kStreamUnroll;     // float4 per tile
+constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
+constexpr int kMaxRowsPerLaunch = 4096;
+constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path
+
+// Per-row state of one batched selection.  Lives in global memory.
+struct RowState {
+    u64 lo;          // the row's candidates are exactly the components with ck >= lo
+    u32 cand_count;  // how many components have ck >= lo (counted, even beyond capacity)
+    u32 max_key;     // largest key among them
+    u32 out_count;   // entries emitted by the final exact selection
+    u32 flags;
+    u32 ticket;      // sampling CTAs of this row that have finished
+    u32 g_active;    // multi-pass path: still refining this row
+    u64 g_lo;        // multi-pass path: known leading bits of the K-th composite key
+    u32 g_need;      // multi-pass path: entries still to take inside the current bucket
+    u32 g_level;
+};
+
+// Step-wide control block.
+struct Ctrl {
+    int status;        // sticky TK_ERR_* raised on the device
+    u32 rows_general;  // rows the multi-pass path handled in the last selection
+    u32 pad[6];
+};
+
+__device__ __forceinline__ u32 key_of(u32 bits) { return bits & 0x7fffffffu; }
+
+__device__ __forceinline__ u64 composite(u32 key, u32 idx) {
+    return ((u64)key << 32) | (u64)(0xffffffffu - idx);
+}
+
+__device__ __forceinline__ void raise_status(Ctrl* ctrl, int code) {
+    atomicCAS(&ctrl->status, 0, code);
+}
+
+// 16-byte read-only streaming load that does not allocate in L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31; }
+
+// Append the lanes with `pred` to a list whose fill counter is *counter.
+// Every lane of the warp must call.  The counter always advances by the number
+// of appending lanes; entries that would land beyond `cap` are dropped (the
+// caller detects that from the counter).  Returns the ballot.
+__device__ __forceinline__ u32 warp_append(bool pred, u32 idx, u32 bits, u32* counter,
+                                           uint2* list, u32 cap) {
+    u32 m = __ballot_sync(0xffffffffu, pred);
+    if (m == 0) return 0;
+    u32 lane = lane_id();
+    u32 base = 0;
+    int leader = __ffs(m) - 1;
+    if ((int)lane == leader) base = atomicAdd(counter, (u32)__popc(m));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (pred) {
+        u32 slot = base + (u32)__popc(m & ((1u << lane) - 1u));
+        if (slot < cap) list[slot] = make_uint2(idx, bits);
+    }
+    return m;
+}
+
+// Inclusive scan of one u32 per thread over the whole block (blockDim.x a
+// multiple of 32, at most 1024).  `scratch` holds 33 words.  Returns the
+// inclusive prefix; *total receives the block sum.
+__device__ __forceinline__ u32 block_inclusive_scan(u32 v, u32* scratch, u32* total) {
+    u32 lane = lane_id(), warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    u32 x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        u32 y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= (u32)o) x += y;
+    }
+    __syncthreads();  // protects scratch against a previous use
+    if (lane == 31) scratch[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+        u32 w = lane < nwarps ? scratch[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u32 y = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= (u32)o) w += y;
+        }
+        if (lane < nwarps) scratch[lane] = w;
+        if (lane == 31) scratch[32] = w;
+    }
+    __syncthreads();
+    if (warp > 0) x += scratch[warp - 1];
+    *total = scratch[32];
+    return x;
+}
+
+// Given a histogram hist[0..nb) in shared memory and 1 <= need <= sum(hist),
+// find the bucket b that holds the need-th entry counted from the TOP bucket
+// downwards, and `above` = entries in buckets > b.  All threads call; the
+// results are returned to every thread.  `res` holds 2 words, `scratch` 33.
+template <int PER>
+__device__ __forceinline__ void find_bucket(const u32* hist, int nb, u32 need, u32* scratch,
+                                            u32* res, u32* b_out, u32* above_out) {
+    // thread t owns the PER buckets nb-1-PER*t ... nb-PER-PER*t (descending)
+    int top = nb - 1 - PER * (int)threadIdx.x;
+    u32 local = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        int b = top - i;
+        if (b >= 0) local += hist[b];
+    }
+    u32 total;
+    u32 incl = block_inclusive_scan(local, scratch, &total);
+    u32 excl = incl - local;
+    if (excl < need && need <= incl) {
+        u32 run = excl;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            int b = top - i;
+            if (b >= 0) {
+                u32 h = hist[b];
+                if (run < need && need <= run + h) { res[0] = (u32)b; res[1] = run; }
+                run += h;
+            }
+        }
+    }
+    __syncthreads();
+    *b_out = res[0];
+    *above_out = res[1];
+    __syncthreads();
+}
+
+}  // namespace tk

@@ -1,0 +1,523 @@
+// Batched exact Top_K selection (Section 1's compressor; the uplink and downlink
+// steps of Algorithm 1/2) as four kernels:
+//
+//   predict_kernel   reads a small strided sample of every row and sets a
+//                    conservative lower bound `lo` on the K-th composite key
+//   filter_kernel    the one streaming pass over all rows*d values: appends every
+//                    component with ck >= lo to the row's candidate list and
+//                    counts them exactly
+//   general_kernel   verification + exact fallback.  A row whose count is below
+//                    K or above the list capacity (or every row, when no
+//                    prediction was made) gets its bound from full-row radix
+//                    histograms (11+11+9 key bits, then 11+11+10 index bits, as
+//                    far as needed) and is filtered again.  Exits at once when
+//                    every row verified.
+//   select_kernel    one thread-block cluster per row: range-adaptive radix
+//                    select of the K largest composite keys among the
+//                    candidates, then emission of exactly K entries
+//
+// The result is always the exact Top_K; the sample only decides how many
+// passes over the data it takes.
+#pragma once
+
+#include "common.cuh"
+
+namespace tk {
+
+// ---------------------------------------------------------------------------
+// predict: sample -> lower bound
+// ---------------------------------------------------------------------------
+// Each of the kSampleSlots threads of a row reads `spt` groups of 8 consecutive
+// values spread evenly over the row and keeps the largest key it saw.  The last
+// CTA of the row to finish takes the `rank`-th largest of these maxima as the
+// bound: at least `rank` sampled values are >= it, so it is never above the
+// rank-th largest sampled value.
+__global__ void __launch_bounds__(kPredictThreads)
+predict_kernel(const float* __restrict__ x, int64_t d, int spt, u32 groups, u32 rank,
+               RowState* rs, u32* smax) {
+    __shared__ u32 sh_hist[256];
+    __shared__ u32 sh_vals[kSampleSlots];
+    __shared__ u32 sh_sel[3];
+    const int row = blockIdx.y;
+    const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;
+    const float* xr = x + (size_t)row * (size_t)d;
+    u32 mx = 0;
+    for (int k = 0; k < spt; ++k) {
+        u64 g = (u64)t + (u64)k * kSampleSlots;
+        u64 e = (g * (u64)(d - 8)) / (u64)(groups - 1);
+        e &= ~7ull;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) mx = max(mx, key_of(__float_as_uint(__ldg(xr + e + c))));
+    }
+    smax[(size_t)row * kSampleSlots + t] = mx;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) sh_sel[0] = atomicAdd(&rs[row].ticket, 1u);
+    __syncthreads();
+    if (sh_sel[0] != kPredictCtas - 1) return;
+    __threadfence();
+
+    // last CTA of the row: rank-th largest of the kSampleSlots maxima, by radix select
+    const volatile u32* vm = smax + (size_t)row * kSampleSlots;
+    for (int i = threadIdx.x; i < kSampleSlots; i += kPredictThreads) sh_vals[i] = vm[i];
+    u32 prefix = 0, need = rank;
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = pass < 3 ? 23 - 8 * pass : 0;
+        const int nb = pass < 3 ? 256 : 128;
+        const int hs = pass < 3 ? shift + 8 : 7;  // bits above this digit
+        if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < kSampleSlots; i += kPredictThreads) {
+            u32 v = sh_vals[i];
+            if ((v >> hs) == (prefix >> hs) || pass == 0)
+                atomicAdd(&sh_hist[(v >> shift) & (u32)(nb - 1)], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            u32 run = 0;
+            int b = nb - 1;
+            for (; b > 0; --b) {
+                if (run + sh_hist[b] >= need) break;
+                run += sh_hist[b];
+            }
+            sh_sel[1] = (u32)b;
+            sh_sel[2] = run;
+        }
+        __syncthreads();
+        prefix |= sh_sel[1] << shift;
+        need -= sh_sel[2];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        RowState* r = rs + row;
+        r->lo = (u64)prefix << 32;
+        r->cand_count = 0;
+        r->max_key = 0;
+        r->out_count = 0;
+        r->flags = 0;
+        r->ticket = 0;
+        r->g_active = 0;
+    }
+}
+
+// No prediction: mark every row for the multi-pass path.
+__global__ void reset_rows_kernel(RowState* rs, int rows) {
+    int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) {
+        rs[r].lo = ~0ull;
+        rs[r].cand_count = 0;
+        rs[r].max_key = 0;
+        rs[r].out_count = 0;
+        rs[r].flags = kRowGeneral;
+        rs[r].ticket = 0;
+        rs[r].g_active = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// filter: the streaming pass
+// ---------------------------------------------------------------------------
+// Geometry of one row: `head` scalar components up to the first 16-byte
+// boundary, then nv float4, then `tail` scalars.
+struct RowGeom {
+    const float* base;
+    const uint4* vec;
+    u32 head, tail;
+    u32 nv;
+};
+
+__device__ __forceinline__ RowGeom row_geom(const float* x, int row, int64_t d) {
+    RowGeom g;
+    g.base = x + (size_t)row * (size_t)d;
+    u32 mis = (u32)(((uintptr_t)g.base >> 2) & 3u);
+    u32 head = (4u - mis) & 3u;
+    if ((int64_t)head > d) head = (u32)d;
+    g.head = head;
+    g.nv = (u32)((d - head) >> 2);
+    g.tail = (u32)(d - head - 4 * (int64_t)g.nv);
+    g.vec = reinterpret_cast<const uint4*>(g.base + head);
+    return g;
+}
+
+// One component in the rare path: append if ck >= lo.
+__device__ __forceinline__ void consider(bool live, u32 idx, u32 bits, u64 lo, RowState* rs,
+                                         uint2* cand, u32 cap) {
+    u32 k = key_of(bits);
+    bool pred = live && composite(k, idx) >= lo;
+    u32 m = warp_append(pred, idx, bits, &rs->cand_count, cand, cap);
+    if (m) {
+        u32 wm = __reduce_max_sync(0xffffffffu, pred ? k : 0u);
+        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&rs->max_key, wm);
+    }
+}
+
+// Process tile `tile` (kTileVecs float4) of a row.  All threads of the CTA call.
+__device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, RowState* rs,
+                                            uint2* cand, u32 cap) {
+    const u32 tk = (u32)(lo >> 32);
+    const u32 j0 = tile * kTileVecs + threadIdx.x;
+    uint4 v[kStreamUnroll];
+    bool inb[kStreamUnroll];
+    const bool full = (u64)(tile + 1) * kTileVecs <= (u64)g.nv;
+    if (full) {
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            v[u] = ld_stream(g.vec + j0 + u * kStreamThreads);
+            inb[u] = true;
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            u32 j = j0 + u * kStreamThreads;
+            inb[u] = j < g.nv;
+            v[u] = inb[u] ? ld_stream(g.vec + j) : make_uint4(0, 0, 0, 0);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+        u32 m = max(max(key_of(v[u].x), key_of(v[u].y)), max(key_of(v[u].z), key_of(v[u].w)));
+        bool hit = inb[u] && m >= tk;
+        if (__any_sync(0xffffffffu, hit)) {
+            u32 i0 = g.head + 4u * (j0 + u * kStreamThreads);
+            consider(hit, i0 + 0, v[u].x, lo, rs, cand, cap);
+            consider(hit, i0 + 1, v[u].y, lo, rs, cand, cap);
+            consider(hit, i0 + 2, v[u].z, lo, rs, cand, cap);
+            consider(hit, i0 + 3, v[u].w, lo, rs, cand, cap);
+        }
+    }
+    if (tile == 0 && threadIdx.x < 32 && (g.head | g.tail)) {
+        u32 lane = threadIdx.x;
+        bool live = false;
+        u32 idx = 0;
+        if (lane < g.head) { live = true; idx = lane; }
+        else if (lane >= 8 && lane - 8 < g.tail) { live = true; idx = g.head + 4u * g.nv + (lane - 8); }
+        u32 bits = live ? __float_as_uint(__ldg(g.base + idx)) : 0u;
+        consider(live, idx, bits, lo, rs, cand, cap);
+    }
+}
+
+__global__ void __launch_bounds__(kStreamThreads)
+filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowState* rs,
+              uint2* cand, u32 cap) {
+    const u32 total = (u32)rows * tpr;
+    int cur = -1;
+    RowGeom g;
+    u64 lo = 0;
+    for (u32 t = blockIdx.x; t < total; t += gridDim.x) {
+        int row = (int)(t / tpr);
+        u32 tile = t - (u32)row * tpr;
+        if (row != cur) {
+            cur = row;
+            g = row_geom(x, row, d);
+            lo = rs[row].lo;
+        }
+        if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
+        filter_tile(g, tile, lo, rs + row, cand + (size_t)row * cap, cap);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// general: verification and the exact multi-pass path (cooperative launch)
+// ---------------------------------------------------------------------------
+// Refinement levels over the 63-bit composite key: {shift, bits}.
+__device__ __constant__ int kLevelShift[6] = {52, 41, 32, 21, 10, 0};
+__device__ __constant__ int kLevelBits[6] = {11, 11, 9, 11, 11, 10};
+
+__device__ __forceinline__ void hist_component(bool live, u32 idx, u32 bits, int level, int shift,
+                                               int nbits, u64 lo, u32* sh_hist) {
+    if (!live) return;
+    u32 k = key_of(bits);
+    if (level == 0) {
+        atomicAdd(&sh_hist[k >> 20], 1u);
+        return;
+    }
+    // cheap test on the key's known leading bits first
+    int top = shift + nbits;  // bits above this level's digit are fixed by lo
+    int kshift = top >= 32 ? top - 32 : 0;
+    if (((k ^ (u32)(lo >> 32)) >> kshift) != 0 && kshift < 32) return;
+    u64 ck = composite(k, idx);
+    if ((ck >> top) != (lo >> top)) return;
+    atomicAdd(&sh_hist[(u32)(ck >> shift) & ((1u << nbits) - 1u)], 1u);
+}
+
+__device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level, u64 lo,
+                                          u32* sh_hist) {
+    const int shift = kLevelShift[level], nbits = kLevelBits[level];
+    const u32 j0 = tile * kTileVecs + threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < kStreamUnroll; ++u) {
+        u32 j = j0 + u * kStreamThreads;
+        if (j < g.nv) {
+            uint4 v = ld_stream(g.vec + j);
+            u32 i0 = g.head + 4u * j;
+            hist_component(true, i0 + 0, v.x, level, shift, nbits, lo, sh_hist);
+            hist_component(true, i0 + 1, v.y, level, shift, nbits, lo, sh_hist);
+            hist_component(true, i0 + 2, v.z, level, shift, nbits, lo, sh_hist);
+            hist_component(true, i0 + 3, v.w, level, shift, nbits, lo, sh_hist);
+        }
+    }
+    if (tile == 0 && threadIdx.x < 32 && (g.head | g.tail)) {
+        u32 lane = threadIdx.x;
+        bool live = false;
+        u32 idx = 0;
+        if (lane < g.head) { live = true; idx = lane; }
+        else if (lane >= 8 && lane - 8 < g.tail) { live = true; idx = g.head + 4u * g.nv + (lane - 8); }
+        u32 bits = live ? __float_as_uint(__ldg(g.base + idx)) : 0u;
+        hist_component(live, idx, bits, level, shift, nbits, lo, sh_hist);
+    }
+}
+
+// Ordered list (in shared memory) of the rows r < rows with pred(r); returns its length.
+template <typename Pred>
+__device__ __forceinline__ int build_row_list(int rows, unsigned short* sh_list, u32* scratch,
+                                              Pred pred) {
+    constexpr int PER = kMaxRowsPerLaunch / kStreamThreads;
+    u32 flags = 0, cnt = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        int r = (int)threadIdx.x * PER + i;
+        if (r < rows && pred(r)) { flags |= 1u << i; ++cnt; }
+    }
+    u32 total;
+    u32 pos = block_inclusive_scan(cnt, scratch, &total) - cnt;
+#pragma unroll
+    for (int i = 0; i < PER; ++i)
+        if (flags & (1u << i)) sh_list[pos++] = (unsigned short)((int)threadIdx.x * PER + i);
+    __syncthreads();
+    return (int)total;
+}
+
+__global__ void __launch_bounds__(kStreamThreads)
+general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr, u32 cap,
+               RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl) {
+    __shared__ u32 sh_hist[kHistBins];
+    __shared__ unsigned short sh_list[kMaxRowsPerLaunch];
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_res[2];
+    cg::grid_group grid = cg::this_grid();
+
+    // Which rows failed verification?  Nothing below modifies a RowState before
+    // the first grid-wide barrier, so every CTA sees the same answer.
+    auto failed = [&](int r) {
+        u32 c = rs[r].cand_count;
+        return (rs[r].flags & kRowGeneral) != 0 || c < K || c > cap;
+    };
+    int nF = build_row_list(rows, sh_list, sh_scratch, failed);
+    if (blockIdx.x == 0 && threadIdx.x == 0) ctrl->rows_general = (u32)nF;
+    if (nF == 0) return;
+
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nF; i += gridDim.x * blockDim.x) {
+        RowState* r = rs + sh_list[i];
+        r->flags |= kRowGeneral;
+        r->g_active = 1;
+        r->g_lo = 0;
+        r->g_need = K;
+        r->g_level = 0;
+    }
+    grid.sync();
+
+    for (int iter = 0; iter < 6; ++iter) {
+        int nA = build_row_list(rows, sh_list, sh_scratch, [&](int r) { return rs[r].g_active != 0; });
+        if (nA == 0) break;
+        // phase A: histograms of the active rows; each CTA takes a contiguous run of tiles
+        {
+            u64 total = (u64)nA * tpr;
+            u64 chunk = (total + gridDim.x - 1) / gridDim.x;
+            u64 t0 = (u64)blockIdx.x * chunk, t1 = min(total, t0 + chunk);
+            int cur = -1, row = 0, level = 0;
+            u64 lo = 0;
+            RowGeom g;
+            for (u64 t = t0; t < t1; ++t) {
+                int li = (int)(t / tpr);
+                u32 tile = (u32)(t - (u64)li * tpr);
+                if (li != cur) {
+                    if (cur >= 0) {
+                        __syncthreads();
+                        for (int b = threadIdx.x; b < kHistBins; b += blockDim.x)
+                            if (sh_hist[b]) atomicAdd(&hist[(size_t)row * kHistBins + b], sh_hist[b]);
+                    }
+                    __syncthreads();
+                    cur = li;
+                    row = sh_list[li];
+                    g = row_geom(x, row, d);
+                    lo = rs[row].g_lo;
+                    level = (int)rs[row].g_level;
+                    for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
+                    __syncthreads();
+                }
+                if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
+                hist_tile(g, tile, level, lo, sh_hist);
+            }
+            if (cur >= 0) {
+                __syncthreads();
+                for (int b = threadIdx.x; b < kHistBins; b += blockDim.x)
+                    if (sh_hist[b]) atomicAdd(&hist[(size_t)row * kHistBins + b], sh_hist[b]);
+            }
+        }
+        grid.sync();
+        // phase B: one CTA per active row picks the bucket of the K-th key
+        for (int li = blockIdx.x; li < nA; li += gridDim.x) {
+            int row = sh_list[li];
+            RowState* r = rs + row;
+            int level = (int)r->g_level;
+            int nb = 1 << kLevelBits[level];
+            __syncthreads();
+            for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) {
+                u32* hp = &hist[(size_t)row * kHistBins + b];
+                sh_hist[b] = __ldcg(hp);
+                *hp = 0;
+            }
+            if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
+            __syncthreads();
+            u32 need = r->g_need, b, above;
+            find_bucket<kHistBins / kStreamThreads>(sh_hist, nb, need, sh_scratch, sh_res, &b, &above);
+            if (threadIdx.x == 0) {
+                if (b == 0xffffffffu) {           // the row holds fewer than `need` entries: cannot happen
+                    raise_status(ctrl, -5);
+                    b = 0; above = 0;
+                    r->g_level = 5;               // ends the refinement below
+                    level = 5;
+                }
+                u64 lo = r->g_lo | ((u64)b << kLevelShift[level]);
+                u32 ge = (K - need) + above + sh_hist[b];  // components with ck >= lo
+                if (ge <= cap || level == 5) {
+                    r->g_active = 0;
+                    r->lo = lo;
+                    r->cand_count = 0;
+                    r->max_key = 0;
+                } else {
+                    r->g_lo = lo;
+                    r->g_need = need - above;
+                    r->g_level = (u32)level + 1;
+                }
+            }
+        }
+        grid.sync();
+    }
+
+    // phase C: filter the failed rows again with their exact bound
+    nF = build_row_list(rows, sh_list, sh_scratch, [&](int r) { return (rs[r].flags & kRowGeneral) != 0; });
+    u64 total = (u64)nF * tpr;
+    int cur = -1, row = 0;
+    u64 lo = 0;
+    RowGeom g;
+    for (u64 t = blockIdx.x; t < total; t += gridDim.x) {
+        int li = (int)(t / tpr);
+        u32 tile = (u32)(t - (u64)li * tpr);
+        if (li != cur) {
+            cur = li;
+            row = sh_list[li];
+            g = row_geom(x, row, d);
+            lo = rs[row].lo;
+        }
+        if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
+        filter_tile(g, tile, lo, rs + row, cand + (size_t)row * cap, cap);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// select: exact K largest composite keys among a row's candidates (one cluster per row)
+// ---------------------------------------------------------------------------
+struct ApplyArgs {
+    float* w;      // if non-NULL: w[idx] -= alpha * val for every emitted entry
+    float alpha;
+};
+
+__global__ void __launch_bounds__(kSelectThreads)
+select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
+              uint2* out, size_t out_stride, ApplyArgs apply, Ctrl* ctrl) {
+    __shared__ u32 sh_hist[kHistBins];
+    __shared__ u32 sh_tot[kHistBins];
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_res[2];
+    cg::cluster_group cluster = cg::this_cluster();
+    const u32 CS = cluster.num_blocks();
+    const u32 rank = cluster.block_rank();
+    const int row = blockIdx.x / CS;
+    RowState* r = rs + row;
+    const u32 C = min(r->cand_count, cap);
+    const u32 Keff = min(K, C);
+    const uint2* list = lists + (size_t)row * list_stride;
+    const u32 first = rank * kSelectThreads + threadIdx.x;
+    const u32 stride = CS * kSelectThreads;
+
+    u64 T = 0;  // emit entries with ck >= T
+    if (C > Keff) {
+        u64 lo = r->lo;
+        u64 hi = ((u64)r->max_key << 32) | 0xffffffffull;
+        if (hi < lo) hi = lo;  // defensive; the candidates then all sit at lo
+        u32 need = Keff;
+        bool found = false;
+        for (int level = 0; level < 8 && !found; ++level) {
+            u64 width = hi - lo;
+            int s = width ? max(0, 64 - __clzll((long long)width) - 11) : 0;
+            int nb = (int)(width >> s) + 1;
+            for (int b = threadIdx.x; b < nb; b += kSelectThreads) sh_hist[b] = 0;
+            if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
+            __syncthreads();
+            for (u32 i = first; i < C; i += stride) {
+                uint2 e = list[i];
+                u64 ck = composite(key_of(e.y), e.x);
+                if (ck >= lo && ck <= hi) atomicAdd(&sh_hist[(u32)((ck - lo) >> s)], 1u);
+            }
+            cluster.sync();
+            for (int b = threadIdx.x; b < nb; b += kSelectThreads) {
+                u32 sum = 0;
+                for (u32 c = 0; c < CS; ++c) sum += cluster.map_shared_rank(sh_hist, c)[b];
+                sh_tot[b] = sum;
+            }
+            __syncthreads();
+            u32 b, above;
+            find_bucket<kHistBins / kSelectThreads>(sh_tot, nb, need, sh_scratch, sh_res, &b, &above);
+            cluster.sync();  // every CTA is done reading its peers' histograms
+            if (b == 0xffffffffu) {
+                if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
+                break;
+            }
+            need -= above;
+            u64 blo = lo + ((u64)b << s);
+            u64 bhi = blo + ((1ull << s) - 1ull);
+            if (bhi > hi) bhi = hi;
+            if (need == sh_tot[b]) { T = blo; found = true; }
+            lo = blo;
+            hi = bhi;
+            __syncthreads();
+        }
+        if (!found) {
+            T = lo;
+            if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
+        }
+    }
+
+    uint2* orow = out + (size_t)row * out_stride;
+    for (u32 i0 = rank * kSelectThreads; i0 < C; i0 += stride) {
+        u32 i = i0 + threadIdx.x;
+        bool pred = false;
+        uint2 e = make_uint2(0, 0);
+        if (i < C) {
+            e = list[i];
+            pred = composite(key_of(e.y), e.x) >= T;
+        }
+        u32 m = __ballot_sync(0xffffffffu, pred);
+        if (m) {
+            u32 lane = lane_id(), base = 0;
+            int leader = __ffs(m) - 1;
+            if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
+            base = __shfl_sync(0xffffffffu, base, leader);
+            if (pred) {
+                u32 slot = base + (u32)__popc(m & ((1u << lane) - 1u));
+                if (slot < Keff) {
+                    orow[slot] = e;
+                    if (apply.w) {
+                        float upd = __fmul_rn(apply.alpha, __uint_as_float(e.y));
+                        apply.w[e.x] = __fsub_rn(apply.w[e.x], upd);
+                    }
+                } else {
+                    raise_status(ctrl, -5);
+                }
+            }
+        }
+    }
+}
+
+}  // namespace tk

@@ -1,0 +1,187 @@
+"""tk_step against the CPU oracle: every stage, every step, on the five workloads."""
+import numpy as np
+import psutil
+import pytest
+import torch
+
+import oracle
+from paper_2209_15203_b200 import binding, workloads as W
+from util import assert_message_equal, assert_values_close, bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def check_step(ctx, wl, w_dev, w_ref, G, alpha, mode, K_down, what):
+    """One step on both sides; returns the oracle's new w."""
+    ctx.tk_step(w_dev, G, alpha, mode)
+    ref = oracle.ref_step(w_ref, G.cpu().numpy(), wl.K_up, K_down, ctx_p(ctx), alpha, mode)
+    st = ctx.tk_status()
+    assert st.device_status == 0
+    # stage 1: the uplink messages
+    uidx, uval = ctx.tk_last_uplink()
+    assert_message_equal(uidx, uval, ref.up_idx, ref.up_val, what + " uplink")
+    # stage 2: the aggregate over the union
+    U = np.nonzero(ref.touched)[0].astype(np.int32)
+    aidx, aval = ctx.tk_last_aggregate()
+    assert st.union_size == U.size <= wl.N * wl.K_up
+    assert np.array_equal(aidx.cpu().numpy(), U), what + " union"
+    assert_values_close(aval.cpu().numpy(), ref.A[U], what + " aggregate")
+    # stage 3: the downlink message
+    midx, mval = ctx.tk_last_downlink()
+    assert np.array_equal(midx.cpu().numpy(), ref.msg_idx), what + " downlink indices"
+    assert_values_close(mval.cpu().numpy(), ref.msg_val, what + " downlink values")
+    # stage 4: the update
+    assert_values_close(w_dev.cpu().numpy(), ref.w, what + " w")
+    # housekeeping: the dense server buffer is back to zero (checked through the next step's union)
+    return ref.w
+
+
+_P = {}
+
+
+def ctx_p(ctx):
+    return _P[id(ctx)]
+
+
+def make_ctx(wl, K_down):
+    p = W.make_p(wl)
+    ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p)
+    _P[id(ctx)] = p.numpy()
+    return ctx
+
+
+def run_workload(wl, steps, modes=None, force_general=False):
+    scale = W.scale_vector(wl, DEV)
+    G = torch.empty((wl.N, wl.d), device=DEV, dtype=torch.float32)
+    for mode in (modes or wl.modes):
+        for K_down in wl.K_down:
+            ctx = make_ctx(wl, K_down)
+            ctx.tk_set_force_general(force_general)
+            w_dev = W.make_w(wl, DEV)
+            w_ref = w_dev.cpu().numpy()
+            for s in range(steps):
+                W.make_grads(wl, s, DEV, out=G, scale=scale)
+                what = "config%d mode=%d K_down=%d step=%d" % (wl.cid, mode, K_down, s)
+                w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, mode, K_down, what)
+            ctx.close()
+
+
+def test_hand_computed_iteration():
+    G = np.array([[1, -8, 0.5, 3, 0, -2, 4, 0.25], [-6, 2, 2, 1, 0, 5, -0.5, 3], [4, 4, -4, 1, 2, 0, 6, -1]],
+                 np.float32)
+    p = torch.tensor([0.5, 0.25, 0.25])
+    for mode, expect in ((1, [1, 3, 1, 1, 1, 1, -0.75, 1]), (0, [1.25, 3, 1, 1, 1, 0.375, -0.75, 1])):
+        ctx = binding.Context(8, 3, 2, 2, p)
+        w = torch.ones(8, device=DEV)
+        ctx.tk_step(w, torch.from_numpy(G).to(DEV), 0.5, mode)
+        assert ctx.tk_status().device_status == 0
+        assert w.cpu().tolist() == expect
+
+
+def test_config1_full_size_all_steps_both_modes():
+    wl = W.workload(1)
+    run_workload(wl, wl.steps)
+
+
+@pytest.mark.parametrize("cid,d", [(2, 1_170_003), (3, 1_280_001), (4, 1_170_000), (5, 3_100_002)])
+def test_scaled_configs_every_step(cid, d):
+    wl = W.workload(cid, d=d)
+    run_workload(wl, 3)
+
+
+def test_scaled_configs_forced_general_path():
+    run_workload(W.workload(2, d=600_001, N=4), 2, force_general=True)
+    run_workload(W.workload(4, d=500_000, N=6), 2, force_general=True)
+
+
+def test_kdown_larger_than_union_pads_with_zero_entries():
+    wl = W.workload(4, d=400_000, N=4)          # K_up = 40, union <= 160; K_down = 4000 > |U|
+    assert wl.K_down[-1] > wl.N * wl.K_up
+    run_workload(wl, 2)
+
+
+def test_set_kdown_between_steps():
+    wl = W.workload(2, d=300_000, N=3)
+    ctx = make_ctx(wl, wl.K_up)
+    w_dev = W.make_w(wl, DEV)
+    w_ref = w_dev.cpu().numpy()
+    for s, kd in enumerate((wl.K_up, 7, 3 * wl.K_up, 1)):
+        ctx.tk_set_kdown(kd)
+        G = W.make_grads(wl, s, DEV)
+        w_ref = check_step(ctx, wl, w_dev, w_ref, G, 0.05, 1, kd, "set_kdown %d" % kd)
+
+
+def test_cancelling_workers_and_zero_weights():
+    d, K = 50_000, 64
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal(d).astype(np.float32)
+    G = np.stack([g, -g, g * 0.5, rng.standard_normal(d).astype(np.float32)])
+    for p in ([0.25, 0.25, 0.25, 0.25], [0.5, 0.5, 0.0, 0.0], [0.0, 0.0, 0.0, 1.0]):
+        pt = torch.tensor(p)
+        for mode in (0, 1):
+            ctx = binding.Context(d, 4, K, K, pt)
+            _P[id(ctx)] = pt.numpy()
+            wl = W.workload(1, d=d)
+            wl = wl.__class__(**{**wl.__dict__, "N": 4, "K_up": K, "K_down": (K,)})
+            w_dev = torch.zeros(d, device=DEV)
+            check_step(ctx, wl, w_dev, np.zeros(d, np.float32), torch.from_numpy(G).to(DEV), 1.0, mode, K,
+                       "cancel p=%s mode=%d" % (p, mode))
+
+
+def test_step_host_matches_device_step():
+    wl = W.workload(2, d=500_000, N=4)
+    G = W.make_grads(wl, 0, DEV)
+    w0 = W.make_w(wl, DEV)
+    ctx = make_ctx(wl, wl.K_up)
+    w_dev = w0.clone()
+    ctx.tk_step(w_dev, G, 0.1, 1)
+    w_host = w0.cpu().pin_memory()
+    ctx.tk_step_host(w_host, G.cpu().pin_memory(), 0.1, 1)
+    assert torch.equal(w_host, w_dev.cpu())
+
+
+def test_same_input_twice_gives_identical_bytes():
+    wl = W.workload(3, d=900_000, N=8)
+    G = W.make_grads(wl, 0, DEV)
+    outs = []
+    for _ in range(2):
+        ctx = make_ctx(wl, wl.K_up)
+        w = W.make_w(wl, DEV)
+        ctx.tk_step(w, G, 0.1, 1)
+        i, v = ctx.tk_last_downlink()
+        outs.append((w.clone(), i.clone(), v.clone()))
+    assert torch.equal(outs[0][0].view(torch.int32), outs[1][0].view(torch.int32))
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2].view(torch.int32), outs[1][2].view(torch.int32))
+
+
+def test_bad_arguments_are_rejected():
+    wl = W.workload(1, d=1000)
+    ctx = make_ctx(wl, 10)
+    w = torch.zeros(1000, device=DEV)
+    G = torch.zeros((4, 1000), device=DEV)
+    with pytest.raises(binding.TkError):
+        ctx.tk_step(w, G, float("nan"), 1)
+    with pytest.raises(binding.TkError):
+        ctx.tk_step(w, G, 0.1, 2)
+    with pytest.raises(binding.TkError):
+        ctx.tk_set_kdown(1001)
+    with pytest.raises(binding.TkError):
+        binding.Context(1000, 4, 10, 10, torch.tensor([0.5, -0.1, 0.3, 0.3]))
+
+
+# ---- full sizes, in the launch configuration the benchmark times ----
+
+def _host_can_hold(wl):
+    need = wl.N * wl.d * 4 * 2 + min(wl.N, oracle.ref.default_threads()) * wl.d * 16 + wl.d * 40
+    return psutil.virtual_memory().available > need * 1.2
+
+
+@pytest.mark.parametrize("cid,steps", [(2, 2), (3, 1), (4, 1), (5, 1)])
+def test_full_size_configs(cid, steps):
+    wl = W.workload(cid)
+    if not _host_can_hold(wl):
+        pytest.skip("not enough host memory for the oracle at this size")
+    if cid == 4:
+        wl = wl.__class__(**{**wl.__dict__, "K_down": (wl.K_down[0], wl.K_down[2])})
+    run_workload(wl, steps, modes=(1,))
