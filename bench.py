@@ -1,0 +1,300 @@
+#!/usr/bin/env python
+"""Benchmark of one bidirectional top_K step (uplink select, ordered aggregation,
+downlink select, update) through the C ABI, on the largest workload.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+Prints one JSON line.  `value` is gradient elements per second (N*d per step,
+summed over GPUs) with the gradients already in HBM; `e2e` is the same metric
+through tk_step_host with pinned host buffers (copies inside the timed region);
+`roofline` is the streaming selection kernel against the measured HBM copy
+bandwidth; `cpu_baseline` is the CPU oracle on the host cores.  With more than
+one GPU every rank runs an independent replica of the workload (the path has
+no exchange between GPUs).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2209_15203_b200 import workloads as W  # noqa: E402
+
+METRIC = "gradient elements/sec per bidirectional top_K step"
+UNIT = "elements/s"
+NOMINAL_HBM_BPS = 8e12
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch on this workload,
+# from the ncu capture summarised under profiles/ (None until captured / after the kernel changed)
+FILTER_TRAFFIC_BYTES = None
+
+
+def measured_hbm_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x10: "sync_boost", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self.stop_flag = False
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def b_min_bytes(wl, k_apply):
+    return 4 * wl.N * wl.d + 24 * wl.N * wl.K_up + 16 * k_apply
+
+
+def run_reference(args, rank, world):
+    """The CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import oracle
+    wl_full = W.workload(args.config)
+    threads = min(wl_full.N, oracle.ref.default_threads())
+    total_steps = args.steps + args.warmup
+    # a full step of the largest workload costs the oracle roughly 2e-8 s per element on 8 cores;
+    # shrink d so that the whole run stays within a few minutes
+    budget = 150.0 / max(1, total_steps)
+    d = wl_full.d
+    est = 2.0e-8 * wl_full.N * d
+    if est > budget:
+        d = max(200_000, int(d * budget / est) // 1000 * 1000)
+    wl = W.workload(args.config, d=d)
+    p = W.make_p(wl).numpy()
+    scale = W.scale_vector(wl, "cpu")
+    w = W.make_w(wl, "cpu").numpy()
+    K_down = wl.K_down[0]
+    times = []
+    for s in range(total_steps):
+        G = W.make_grads(wl, s, "cpu", scale=scale).numpy()
+        t0 = time.perf_counter()
+        res = oracle.ref_step(w, G, wl.K_up, K_down, p, wl.alpha, 1, nthreads=threads, want_dense=False)
+        t1 = time.perf_counter()
+        w = res.w
+        if s >= args.warmup:
+            times.append(t1 - t0)
+    t = sum(times)
+    value = wl.N * wl.d * len(times) / t
+    sample = "config %d recipe at d=%d of %d (N=%d, K=%d), full steps" % (wl.cid, wl.d, wl_full.d, wl.N, wl.K_up)
+    cfg = W.describe(wl_full)
+    cfg["sampled_d"] = wl.d
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": cfg,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch.distributed as dist
+    from paper_2209_15203_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    warmup = max(args.warmup, 3)
+    wl = W.workload(args.config)
+    K_down = wl.K_down[0]
+    p = W.make_p(wl)
+    ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p)
+    scale = W.scale_vector(wl, dev)
+    nbuf = max(1, min(args.steps, 8))
+    bufs = [W.make_grads(wl, s, dev, scale=scale) for s in range(nbuf)]
+    del scale
+    w = W.make_w(wl, dev)
+    mode = binding.TK_MODE_BIDIR
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for s in range(warmup):
+        ctx.tk_step(w, bufs[s % nbuf], wl.alpha, mode)
+    st = ctx.tk_status()
+    ctx.tk_set_profile(True)
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.tk_launch_count()
+    barrier()
+    sampler.start()
+    ev0.record()
+    for s in range(args.steps):
+        ctx.tk_step(w, bufs[s % nbuf], wl.alpha, mode)
+    ev1.record()
+    barrier()
+    sampler.stop_flag = True
+    ms = ev0.elapsed_time(ev1)
+    launches = ctx.tk_launch_count() - launches0
+    st = ctx.tk_status()
+    sampler.join(timeout=2.0)
+    ctx.tk_set_profile(False)
+
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    elems = wl.N * wl.d
+    value = world * elems * args.steps / (ms_max * 1e-3)
+    ms_per_step = ms_max / args.steps
+
+    # roofline of the dominant kernel (the streaming selection pass)
+    peak, peak_kind = measured_hbm_gbs()
+    roof = None
+    if st.select_samples > 0:
+        k_ms = st.select_ms_sum / st.select_samples
+        achieved = 4.0 * elems / (k_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "kernel": "filter_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": FILTER_TRAFFIC_BYTES,
+                "algorithmic_bytes": 4 * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
+
+    # end to end through tk_step_host: pinned host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        g_host = torch.empty((wl.N, wl.d), dtype=torch.float32, pin_memory=True)
+        g_host.copy_(bufs[0])
+        w_host = torch.empty(wl.d, dtype=torch.float32, pin_memory=True)
+        w_host.copy_(w)
+        n_e2e = max(1, min(args.steps, 5))
+        ctx.tk_step_host(w_host, g_host, wl.alpha, mode)          # warm-up: allocates the staging buffers
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            ctx.tk_step_host(w_host, g_host, wl.alpha, mode)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * elems * n_e2e / float(tt.item()), "unit": UNIT,
+               "h2d_bytes_per_step": 4 * (elems + wl.d), "d2h_bytes_per_step": 4 * wl.d, "steps": n_e2e,
+               "ms_per_step": 1e3 * float(tt.item()) / n_e2e}
+        del g_host, w_host
+
+    # the CPU oracle on this host's cores: one full step of the same workload (rank 0, single GPU only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        threads = min(wl.N, oracle.ref.default_threads())
+        G = bufs[0].cpu().numpy()
+        w_cpu = w.cpu().numpy()
+        t0 = time.perf_counter()
+        oracle.ref_step(w_cpu, G, wl.K_up, K_down, p.numpy(), wl.alpha, 1, nthreads=threads, want_dense=False)
+        dt = time.perf_counter() - t0
+        cpu = {"value": elems / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "1 full step of config %d (N=%d rows of d=%d), %.1f s" % (wl.cid, wl.N, wl.d, dt)}
+
+    if rank == 0:
+        cfg = W.describe(wl)
+        cfg.update({"mode": "bidirectional", "cold_inputs": "each step reads a %d MB gradient tensor (>> L2), "
+                    "%d distinct tensors cycled" % (4 * elems // 10 ** 6, nbuf),
+                    "parallelism": "replicas x%d" % world})
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
+            "hbm_frac_of_8TBps": b_min_bytes(wl, K_down) / (ms_per_step * 1e-3) / NOMINAL_HBM_BPS,
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+            "stats": {"rows_general": st.rows_general, "union_size": st.union_size,
+                      "cand_min": st.cand_min, "cand_max": st.cand_max, "device_status": st.device_status},
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
