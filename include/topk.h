@@ -53,7 +53,8 @@ enum {
     TK_ERR_ALLOC = -2,    /* workspace too small / allocation failed */
     TK_ERR_CUDA = -3,     /* a CUDA runtime call failed */
     TK_ERR_TIMEOUT = -4,  /* a bounded device-side wait expired */
-    TK_ERR_INTERNAL = -5  /* a device-side consistency check failed */
+    TK_ERR_INTERNAL = -5, /* a device-side consistency check failed */
+    TK_ERR_TOO_LARGE = -6 /* the problem does not fit the built-in scratch of tk_topk_noalloc */
 };
 
 enum {
@@ -125,6 +126,44 @@ int tk_step_host(tk_ctx* ctx, float* w_host, const float* grads_host, float alph
  */
 int tk_topk(tk_ctx* ctx, const float* x_dev, int32_t rows, int64_t d, int64_t K,
             int32_t* idx_out_dev, float* val_out_dev);
+
+/*
+ * tk_topk for callers that must not allocate.  (The paper has no counterpart:
+ * this is a packaging variant of the call above, not another operation.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or
+ * impossible — a plugin that lives inside somebody else's memory budget, a
+ * real-time loop that may not take the allocator's locks or the implicit
+ * device-wide synchronisation of cudaFree, a process whose memory was handed
+ * out in full at start-up.  tk_topk would call cudaMalloc the first time (and
+ * whenever a larger problem arrives); this entry point never calls cudaMalloc,
+ * cudaFree or any other allocating routine.  All of its scratch memory (row
+ * states, histograms, candidate lists, sort buffers) lives in one array of
+ * TK_NOALLOC_SCRATCH_BYTES bytes that is part of the library image: every GPU
+ * that loads the library holds that much memory until the process exits,
+ * whether or not this function is ever called.
+ *
+ *   x_dev, rows, d, K, idx_out_dev, val_out_dev   exactly as for tk_topk; the
+ *               caller still provides the input and both outputs
+ *   cuda_stream a cudaStream_t (NULL = the legacy default stream)
+ *
+ * Limits and rules
+ *   - The scratch a problem needs grows with rows*(min(d, 4K + 8192) + 2K) *
+ *     8 bytes plus about 25 KB per row.  If that exceeds the array the call
+ *     returns TK_ERR_TOO_LARGE and does nothing (for example rows = 8 with
+ *     K = 4096 fits; K beyond about 80,000 does not fit even for one row).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and queries launch limits.  Make that first call
+ *     before starting any stream capture.
+ *   - All calls share the one array, which keeps whatever the previous call
+ *     left in it; the function clears the parts that must start at zero.  Two
+ *     calls whose GPU work overlaps (different streams, different host
+ *     threads) race on it: serialise them.
+ * Asynchronous; results are identical to tk_topk's.
+ */
+#define TK_NOALLOC_SCRATCH_BYTES (4u << 20)
+int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
+                    float* val_out_dev, void* cuda_stream);
 
 /* Change K_downlink of an existing context (1 <= K_down <= d). */
 int tk_set_kdown(tk_ctx* ctx, int64_t K_down);

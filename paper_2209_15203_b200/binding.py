@@ -19,7 +19,7 @@ from . import build as _build
 TK_MODE_UNI = 0
 TK_MODE_BIDIR = 1
 
-EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_set_kdown",
+EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
            "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
@@ -65,6 +65,8 @@ def load(build_if_missing: bool = True):
     lib.tk_step.argtypes = [vp, vp, vp, f32, ctypes.c_int]
     lib.tk_step_host.argtypes = [vp, vp, vp, f32, ctypes.c_int]
     lib.tk_topk.argtypes = [vp, vp, i32, i64, i64, vp, vp]
+    lib.tk_topk_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, vp]
+    lib.tk_topk_noalloc.restype = ctypes.c_int
     lib.tk_set_kdown.argtypes = [vp, i64]
     lib.tk_last_uplink.argtypes = [vp, vp, vp]
     lib.tk_last_aggregate.argtypes = [vp, vp, vp, ctypes.POINTER(i64)]
@@ -211,6 +213,21 @@ def tk_topk(x: torch.Tensor, K: int, ctx: Optional[Context] = None) -> Tuple[tor
     if x.dim() == 1:
         return idx[0], val[0]
     return idx, val
+
+
+def tk_topk_noalloc(x: torch.Tensor, K: int, idx: torch.Tensor, val: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Top_K of every row of x into the caller's idx / val tensors without any device
+    allocation: the library's scratch is a fixed array inside the library image (see
+    include/topk.h for its size, the set-up done by the first call and the rule that
+    overlapping calls race).  Raises TkError(-6) when the problem does not fit."""
+    x2 = x if x.dim() == 2 else x.reshape(1, -1)
+    rows, d = x2.shape
+    assert idx.numel() == rows * K and val.numel() == rows * K
+    with torch.cuda.device(x.device):
+        s = stream if stream is not None else torch.cuda.current_stream(x.device)
+        _check(load().tk_topk_noalloc(_dev(x2, torch.float32), rows, d, K, _dev(idx, torch.int32),
+                                      _dev(val, torch.float32), s.cuda_stream), "tk_topk_noalloc")
 
 
 def tk_release_scratch() -> None:

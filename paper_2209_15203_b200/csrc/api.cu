@@ -658,6 +658,49 @@ void tk_release_scratch(void) {
     }
 }
 
+// ---- tk_topk without allocation ----------------------------------------------------------------
+// The scratch of tk_topk_noalloc.  In host code this name is only a handle for
+// cudaGetSymbolAddress: the kernels get the device address looked up below.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TK_NOALLOC_SCRATCH_BYTES];
+static char* g_noalloc_addr[64];  // device address of the array, per device; NULL until looked up
+
+int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
+                    float* val_out_dev, void* cuda_stream) {
+    if (!aligned4(x_dev) || !aligned4(idx_out_dev) || !aligned4(val_out_dev)) return TK_ERR_INVALID;
+    if (rows < 1 || d < 1 || d >= ((int64_t)1 << 31) || K < 1 || K > d) return TK_ERR_INVALID;
+    // size check first, in 64-bit arithmetic that cannot wrap for any accepted rows/d/K
+    if ((double)rows * ((double)candidate_capacity(d, K) + 2.0 * (double)K) * 8.0 > (double)TK_NOALLOC_SCRATCH_BYTES)
+        return TK_ERR_TOO_LARGE;
+    SelectLayout SL = select_layout(rows, d, K);
+    SortLayout QL = sort_layout(rows, K);
+    size_t off_ctrl = SL.bytes + QL.bytes;
+    if (off_ctrl + align_up(sizeof(Ctrl)) > (size_t)TK_NOALLOC_SCRATCH_BYTES) return TK_ERR_TOO_LARGE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
+    if (!g_noalloc_addr[dev]) {  // set-up, once per device, with that device current
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return TK_ERR_CUDA;
+        }
+        g_noalloc_addr[dev] = (char*)ptr;
+    }
+    char* base = g_noalloc_addr[dev];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    SelectBufs b = bind(SL, base);
+    Ctrl* ctrl = (Ctrl*)(base + off_ctrl);
+    // the array still holds the previous call's data: clear what the kernels expect to be zero
+    if (cudaMemsetAsync(b.rs, 0, (size_t)rows * sizeof(RowState), s) != cudaSuccess ||
+        cudaMemsetAsync(b.hist, 0, (size_t)rows * kHistBins * sizeof(u32), s) != cudaSuccess ||
+        cudaMemsetAsync(ctrl, 0, sizeof(Ctrl), s) != cudaSuccess)
+        return TK_ERR_CUDA;
+    int64_t launches = 0;
+    int rc = run_select(s, x_dev, rows, d, K, b, ctrl, false, nullptr, nullptr, &launches);
+    if (rc != TK_OK) return rc;
+    return run_sort(s, b.out, (size_t)K, nullptr, 0, (u32)K, rows, d, (uint2*)(base + SL.bytes + QL.off_tmp),
+                    (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, &launches);
+}
+
 const char* tk_strerror(int code) {
     switch (code) {
         case TK_OK: return "ok";
@@ -666,6 +709,7 @@ const char* tk_strerror(int code) {
         case TK_ERR_CUDA: return "CUDA runtime error";
         case TK_ERR_TIMEOUT: return "bounded device-side wait expired";
         case TK_ERR_INTERNAL: return "device-side consistency check failed";
+        case TK_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of tk_topk_noalloc";
         default: return "unknown error";
     }
 }
