@@ -56,11 +56,7 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
     }
     u32 bits = __float_as_uint(acc);
-    u32 m = warp_append(owner, j, bits, &uni->cand_count, U, ucap);
-    if (m) {
-        u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
-        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&uni->max_key, wm);
-    }
+    warp_append(owner, j, bits, &uni->cand_count, U, ucap);
 }
 
 // Start-of-step reset of the union's state and the downlink counter.

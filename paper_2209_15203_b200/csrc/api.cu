@@ -280,7 +280,8 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             TK_LAUNCH_CHECK();
             if (ev0) cudaEventRecord(ev0, stream);
             u64 tiles = (u64)nr * b.tpr;
-            u32 grid = (u32)(tiles < (u64)(di->sms * 4) ? tiles : (u64)(di->sms * 4));
+            u64 resident = (u64)di->sms * kStreamCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
+            u32 grid = (u32)(tiles < resident ? tiles : resident);
             filter_kernel<<<grid, kStreamThreads, 0, stream>>>(xb, nr, d, b.tpr, rs, cand, b.cap);
             TK_LAUNCH_CHECK();
             if (ev1) cudaEventRecord(ev1, stream);

@@ -27,6 +27,7 @@ constexpr int kPredictThreads = 512;
 constexpr int kSampleSlots = kPredictCtas * kPredictThreads;  // per-row sample maxima
 constexpr int kStreamThreads = 512;    // streaming kernels: threads per CTA
 constexpr int kStreamUnroll = 4;       // 16-byte loads in flight per thread
+constexpr int kStreamCtasPerSm = 2;    // filter kernel: resident CTAs per SM (grid = that x SMs)
 constexpr int kTileVecs = kStreamThreads * kStreamUnroll;     // float4 per tile
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 constexpr int kMaxRowsPerLaunch = 4096;
@@ -36,7 +37,7 @@ constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the mult
 struct RowState {
     u64 lo;          // the row's candidates are exactly the components with ck >= lo
     u32 cand_count;  // how many components have ck >= lo (counted, even beyond capacity)
-    u32 max_key;     // largest key among them
+    u32 max_key;     // unused by the kernels (kept for layout stability)
     u32 out_count;   // entries emitted by the final exact selection
     u32 flags;
     u32 ticket;      // sampling CTAs of this row that have finished

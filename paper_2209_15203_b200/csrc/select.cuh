@@ -36,18 +36,38 @@ __global__ void __launch_bounds__(kPredictThreads)
 predict_kernel(const float* __restrict__ x, int64_t d, int spt, u32 groups, u32 rank,
                RowState* rs, u32* smax) {
     __shared__ u32 sh_hist[256];
-    __shared__ u32 sh_vals[kSampleSlots];
     __shared__ u32 sh_sel[3];
     const int row = blockIdx.y;
     const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;
     const float* xr = x + (size_t)row * (size_t)d;
+    const bool vec_ok = (((uintptr_t)xr) & 15u) == 0;  // groups start at multiples of 8 elements
+    const u64 span = (u64)(d - 8), div = (u64)(groups - 1);
     u32 mx = 0;
-    for (int k = 0; k < spt; ++k) {
-        u64 g = (u64)t + (u64)k * kSampleSlots;
-        u64 e = (g * (u64)(d - 8)) / (u64)(groups - 1);
-        e &= ~7ull;
+    for (int k0 = 0; k0 < spt; k0 += 4) {
+        uint4 a[4], b[4];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) mx = max(mx, key_of(__float_as_uint(__ldg(xr + e + c))));
+        for (int u = 0; u < 4; ++u) {
+            a[u] = make_uint4(0, 0, 0, 0);
+            b[u] = make_uint4(0, 0, 0, 0);
+            if (k0 + u < spt) {
+                u64 g = (u64)t + (u64)(k0 + u) * kSampleSlots;
+                u64 e = ((g * span) / div) & ~7ull;
+                if (vec_ok) {
+                    a[u] = ld_stream(reinterpret_cast<const uint4*>(xr + e));
+                    b[u] = ld_stream(reinterpret_cast<const uint4*>(xr + e) + 1);
+                } else {
+                    a[u] = make_uint4(__float_as_uint(__ldg(xr + e)), __float_as_uint(__ldg(xr + e + 1)),
+                                      __float_as_uint(__ldg(xr + e + 2)), __float_as_uint(__ldg(xr + e + 3)));
+                    b[u] = make_uint4(__float_as_uint(__ldg(xr + e + 4)), __float_as_uint(__ldg(xr + e + 5)),
+                                      __float_as_uint(__ldg(xr + e + 6)), __float_as_uint(__ldg(xr + e + 7)));
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            mx = max(mx, max(max(key_of(a[u].x), key_of(a[u].y)), max(key_of(a[u].z), key_of(a[u].w))));
+            mx = max(mx, max(max(key_of(b[u].x), key_of(b[u].y)), max(key_of(b[u].z), key_of(b[u].w))));
+        }
     }
     smax[(size_t)row * kSampleSlots + t] = mx;
     __threadfence();
@@ -59,29 +79,49 @@ predict_kernel(const float* __restrict__ x, int64_t d, int spt, u32 groups, u32 
 
     // last CTA of the row: rank-th largest of the kSampleSlots maxima, by radix select
     const volatile u32* vm = smax + (size_t)row * kSampleSlots;
-    for (int i = threadIdx.x; i < kSampleSlots; i += kPredictThreads) sh_vals[i] = vm[i];
+    u32 mine[kSampleSlots / kPredictThreads];
+#pragma unroll
+    for (int i = 0; i < kSampleSlots / kPredictThreads; ++i) mine[i] = vm[threadIdx.x + i * kPredictThreads];
     u32 prefix = 0, need = rank;
     for (int pass = 0; pass < 4; ++pass) {
         const int shift = pass < 3 ? 23 - 8 * pass : 0;
         const int nb = pass < 3 ? 256 : 128;
         const int hs = pass < 3 ? shift + 8 : 7;  // bits above this digit
         if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
+        if (threadIdx.x == 0) { sh_sel[1] = 0; sh_sel[2] = 0; }
         __syncthreads();
-        for (int i = threadIdx.x; i < kSampleSlots; i += kPredictThreads) {
-            u32 v = sh_vals[i];
-            if ((v >> hs) == (prefix >> hs) || pass == 0)
-                atomicAdd(&sh_hist[(v >> shift) & (u32)(nb - 1)], 1u);
+#pragma unroll
+        for (int i = 0; i < kSampleSlots / kPredictThreads; ++i) {
+            u32 v = mine[i];
+            if ((v >> hs) == (prefix >> hs)) atomicAdd(&sh_hist[(v >> shift) & (u32)(nb - 1)], 1u);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            u32 run = 0;
-            int b = nb - 1;
-            for (; b > 0; --b) {
-                if (run + sh_hist[b] >= need) break;
-                run += sh_hist[b];
+        if (threadIdx.x < 32) {
+            // lane l owns the 8 bins nb-1-8l .. nb-8-8l (descending); bins below 0 do not exist
+            u32 lane = threadIdx.x, local = 0;
+            int top = nb - 1 - 8 * (int)lane;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) if (top - i >= 0) local += sh_hist[top - i];
+            u32 incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                u32 y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= (u32)o) incl += y;
             }
-            sh_sel[1] = (u32)b;
-            sh_sel[2] = run;
+            u32 total = __shfl_sync(0xffffffffu, incl, 31);
+            u32 want = need <= total ? need : total;  // fewer maxima than rank: take the smallest
+            u32 excl = incl - local;
+            if (want > 0 && excl < want && want <= incl) {
+                u32 run = excl;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (top - i >= 0) {
+                        u32 h = sh_hist[top - i];
+                        if (run < want && want <= run + h) { sh_sel[1] = (u32)(top - i); sh_sel[2] = run; }
+                        run += h;
+                    }
+                }
+            }
         }
         __syncthreads();
         prefix |= sh_sel[1] << shift;
@@ -144,11 +184,7 @@ __device__ __forceinline__ void consider(bool live, u32 idx, u32 bits, u64 lo, R
                                          uint2* cand, u32 cap) {
     u32 k = key_of(bits);
     bool pred = live && composite(k, idx) >= lo;
-    u32 m = warp_append(pred, idx, bits, &rs->cand_count, cand, cap);
-    if (m) {
-        u32 wm = __reduce_max_sync(0xffffffffu, pred ? k : 0u);
-        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&rs->max_key, wm);
-    }
+    warp_append(pred, idx, bits, &rs->cand_count, cand, cap);
 }
 
 // Process tile `tile` (kTileVecs float4) of a row.  All threads of the CTA call.
@@ -196,7 +232,7 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
     }
 }
 
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowState* rs,
               uint2* cand, u32 cap) {
     const u32 total = (u32)rows * tpr;
@@ -423,6 +459,8 @@ struct ApplyArgs {
     float alpha;
 };
 
+constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
+
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
               uint2* out, size_t out_stride, ApplyArgs apply, Ctrl* ctrl) {
@@ -430,6 +468,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     __shared__ u32 sh_tot[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
+    __shared__ u32 sh_max;
     cg::cluster_group cluster = cg::this_cluster();
     const u32 CS = cluster.num_blocks();
     const u32 rank = cluster.block_rank();
@@ -440,12 +479,35 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     const uint2* list = lists + (size_t)row * list_stride;
     const u32 first = rank * kSelectThreads + threadIdx.x;
     const u32 stride = CS * kSelectThreads;
+    const u32 rest = first + kSelectRegs * stride;  // entries from here on are re-read every level
+
+    // this thread's entries first + k*stride, k < kSelectRegs, stay in registers
+    u32 eidx[kSelectRegs], ebits[kSelectRegs];
+#pragma unroll
+    for (int k = 0; k < kSelectRegs; ++k) {
+        u32 i = first + (u32)k * stride;
+        uint2 e = i < C ? list[i] : make_uint2(0xffffffffu, 0u);  // absent: ck = 0
+        eidx[k] = e.x;
+        ebits[k] = e.y;
+    }
 
     u64 T = 0;  // emit entries with ck >= T
     if (C > Keff) {
+        // the largest key bounds the range from above
+        u32 mx = 0;
+#pragma unroll
+        for (int k = 0; k < kSelectRegs; ++k) mx = max(mx, key_of(ebits[k]));
+        for (u32 i = rest; i < C; i += stride) mx = max(mx, key_of(list[i].y));
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (threadIdx.x == 0) sh_max = 0;
+        __syncthreads();
+        if (lane_id() == 0) atomicMax(&sh_max, mx);
+        cluster.sync();
+        mx = 0;
+        for (u32 c = 0; c < CS; ++c) mx = max(mx, *cluster.map_shared_rank(&sh_max, c));
         u64 lo = r->lo;
-        u64 hi = ((u64)r->max_key << 32) | 0xffffffffull;
-        if (hi < lo) hi = lo;  // defensive; the candidates then all sit at lo
+        u64 hi = ((u64)mx << 32) | 0xffffffffull;
+        if (hi < lo) hi = lo;
         u32 need = Keff;
         bool found = false;
         for (int level = 0; level < 8 && !found; ++level) {
@@ -455,7 +517,12 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             for (int b = threadIdx.x; b < nb; b += kSelectThreads) sh_hist[b] = 0;
             if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
             __syncthreads();
-            for (u32 i = first; i < C; i += stride) {
+#pragma unroll
+            for (int k = 0; k < kSelectRegs; ++k) {
+                u64 ck = composite(key_of(ebits[k]), eidx[k]);
+                if (ck >= lo && ck <= hi && eidx[k] != 0xffffffffu) atomicAdd(&sh_hist[(u32)((ck - lo) >> s)], 1u);
+            }
+            for (u32 i = rest; i < C; i += stride) {
                 uint2 e = list[i];
                 u64 ck = composite(key_of(e.y), e.x);
                 if (ck >= lo && ck <= hi) atomicAdd(&sh_hist[(u32)((ck - lo) >> s)], 1u);
@@ -489,8 +556,37 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         }
     }
 
+    // emission: every entry with ck >= T, exactly Keff of them
     uint2* orow = out + (size_t)row * out_stride;
-    for (u32 i0 = rank * kSelectThreads; i0 < C; i0 += stride) {
+    auto emit = [&](bool pred, u32 idx, u32 bits) {
+        u32 m = __ballot_sync(0xffffffffu, pred);
+        if (m == 0) return;
+        u32 lane = lane_id(), base = 0;
+        int leader = __ffs(m) - 1;
+        if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
+        base = __shfl_sync(0xffffffffu, base, leader);
+        if (pred) {
+            u32 slot = base + (u32)__popc(m & ((1u << lane) - 1u));
+            if (slot < Keff) {
+                orow[slot] = make_uint2(idx, bits);
+                if (apply.w) {
+                    float upd = __fmul_rn(apply.alpha, __uint_as_float(bits));
+                    apply.w[idx] = __fsub_rn(apply.w[idx], upd);
+                }
+            } else {
+                raise_status(ctrl, -5);
+            }
+        }
+    };
+    // counts per thread first, so that one atomic per warp covers all register-held entries
+#pragma unroll
+    for (int k = 0; k < kSelectRegs; ++k) {
+        if (__any_sync(0xffffffffu, first + (u32)k * stride < C)) {
+            bool pred = eidx[k] != 0xffffffffu && composite(key_of(ebits[k]), eidx[k]) >= T;
+            emit(pred, eidx[k], ebits[k]);
+        }
+    }
+    for (u32 i0 = rank * kSelectThreads + kSelectRegs * stride; i0 < C; i0 += stride) {
         u32 i = i0 + threadIdx.x;
         bool pred = false;
         uint2 e = make_uint2(0, 0);
@@ -498,25 +594,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             e = list[i];
             pred = composite(key_of(e.y), e.x) >= T;
         }
-        u32 m = __ballot_sync(0xffffffffu, pred);
-        if (m) {
-            u32 lane = lane_id(), base = 0;
-            int leader = __ffs(m) - 1;
-            if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
-            base = __shfl_sync(0xffffffffu, base, leader);
-            if (pred) {
-                u32 slot = base + (u32)__popc(m & ((1u << lane) - 1u));
-                if (slot < Keff) {
-                    orow[slot] = e;
-                    if (apply.w) {
-                        float upd = __fmul_rn(apply.alpha, __uint_as_float(e.y));
-                        apply.w[e.x] = __fsub_rn(apply.w[e.x], upd);
-                    }
-                } else {
-                    raise_status(ctrl, -5);
-                }
-            }
-        }
+        emit(pred, e.x, e.y);
     }
 }
 
