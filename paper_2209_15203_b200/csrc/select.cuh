@@ -179,17 +179,57 @@ __device__ __forceinline__ RowGeom row_geom(const float* x, int row, int64_t d) 
     return g;
 }
 
-// One component in the rare path: append if ck >= lo.
-__device__ __forceinline__ void consider(bool live, u32 idx, u32 bits, u64 lo, RowState* rs,
-                                         uint2* cand, u32 cap) {
-    u32 k = key_of(bits);
-    bool pred = live && composite(k, idx) >= lo;
-    warp_append(pred, idx, bits, &rs->cand_count, cand, cap);
+// Candidates are first collected per warp in shared memory and appended to the
+// row's list in batches: hits cluster in the layers with the largest scale, and
+// one global atomic per hit on the row's single counter would serialise there.
+constexpr int kStageSlots = 64;  // per warp; at least 32
+
+struct WarpStage {
+    uint2* buf;  // this warp's kStageSlots entries
+    u32* n;      // this warp's fill count
+};
+
+__device__ __forceinline__ WarpStage warp_stage(uint2* sh_buf, u32* sh_n) {
+    WarpStage st;
+    u32 warp = threadIdx.x >> 5;
+    st.buf = sh_buf + warp * kStageSlots;
+    st.n = sh_n + warp;
+    return st;
+}
+
+// Append the warp's staged entries to the row's candidate list.  All lanes call.
+__device__ __forceinline__ void stage_flush(const WarpStage& st, RowState* rs, uint2* cand, u32 cap) {
+    u32 n = *st.n;
+    if (n == 0) return;
+    u32 lane = lane_id(), base = 0;
+    if (lane == 0) base = atomicAdd(&rs->cand_count, n);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    for (u32 i = lane; i < n; i += 32)
+        if (base + i < cap) cand[base + i] = st.buf[i];
+    __syncwarp();
+    if (lane == 0) *st.n = 0;
+    __syncwarp();
+}
+
+// One component in the rare path: stage it if ck >= lo.  All lanes call.
+__device__ __forceinline__ void consider(bool live, u32 idx, u32 bits, u64 lo, const WarpStage& st,
+                                         RowState* rs, uint2* cand, u32 cap) {
+    bool pred = live && composite(key_of(bits), idx) >= lo;
+    u32 m = __ballot_sync(0xffffffffu, pred);
+    if (m == 0) return;
+    u32 cnt = (u32)__popc(m);
+    if (*st.n + cnt > kStageSlots) stage_flush(st, rs, cand, cap);
+    u32 n = *st.n;
+    u32 lane = lane_id();
+    if (pred) st.buf[n + (u32)__popc(m & ((1u << lane) - 1u))] = make_uint2(idx, bits);
+    __syncwarp();
+    if (lane == 0) *st.n = n + cnt;
+    __syncwarp();
 }
 
 // Process tile `tile` (kTileVecs float4) of a row.  All threads of the CTA call.
-__device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, RowState* rs,
-                                            uint2* cand, u32 cap) {
+__device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
+                                            RowState* rs, uint2* cand, u32 cap) {
     const u32 tk = (u32)(lo >> 32);
     const u32 j0 = tile * kTileVecs + threadIdx.x;
     uint4 v[kStreamUnroll];
@@ -215,10 +255,10 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
         bool hit = inb[u] && m >= tk;
         if (__any_sync(0xffffffffu, hit)) {
             u32 i0 = g.head + 4u * (j0 + u * kStreamThreads);
-            consider(hit, i0 + 0, v[u].x, lo, rs, cand, cap);
-            consider(hit, i0 + 1, v[u].y, lo, rs, cand, cap);
-            consider(hit, i0 + 2, v[u].z, lo, rs, cand, cap);
-            consider(hit, i0 + 3, v[u].w, lo, rs, cand, cap);
+            consider(hit && key_of(v[u].x) >= tk, i0 + 0, v[u].x, lo, st, rs, cand, cap);
+            consider(hit && key_of(v[u].y) >= tk, i0 + 1, v[u].y, lo, st, rs, cand, cap);
+            consider(hit && key_of(v[u].z) >= tk, i0 + 2, v[u].z, lo, st, rs, cand, cap);
+            consider(hit && key_of(v[u].w) >= tk, i0 + 3, v[u].w, lo, st, rs, cand, cap);
         }
     }
     if (tile == 0 && threadIdx.x < 32 && (g.head | g.tail)) {
@@ -228,13 +268,18 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
         if (lane < g.head) { live = true; idx = lane; }
         else if (lane >= 8 && lane - 8 < g.tail) { live = true; idx = g.head + 4u * g.nv + (lane - 8); }
         u32 bits = live ? __float_as_uint(__ldg(g.base + idx)) : 0u;
-        consider(live, idx, bits, lo, rs, cand, cap);
+        consider(live, idx, bits, lo, st, rs, cand, cap);
     }
 }
 
 __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowState* rs,
               uint2* cand, u32 cap) {
+    __shared__ uint2 sh_buf[(kStreamThreads / 32) * kStageSlots];
+    __shared__ u32 sh_n[kStreamThreads / 32];
+    if (threadIdx.x < kStreamThreads / 32) sh_n[threadIdx.x] = 0;
+    __syncthreads();
+    const WarpStage st = warp_stage(sh_buf, sh_n);
     const u32 total = (u32)rows * tpr;
     int cur = -1;
     RowGeom g;
@@ -243,13 +288,15 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowStat
         int row = (int)(t / tpr);
         u32 tile = t - (u32)row * tpr;
         if (row != cur) {
+            if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
             cur = row;
             g = row_geom(x, row, d);
             lo = rs[row].lo;
         }
         if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile(g, tile, lo, rs + row, cand + (size_t)row * cap, cap);
+        filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
     }
+    if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
 }
 
 // ---------------------------------------------------------------------------
@@ -330,6 +377,8 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
     __shared__ unsigned short sh_list[kMaxRowsPerLaunch];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
+    __shared__ uint2 sh_buf[(kStreamThreads / 32) * kStageSlots];
+    __shared__ u32 sh_n[kStreamThreads / 32];
     cg::grid_group grid = cg::this_grid();
 
     // Which rows failed verification?  Nothing below modifies a RowState before
@@ -433,6 +482,9 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
 
     // phase C: filter the failed rows again with their exact bound
     nF = build_row_list(rows, sh_list, sh_scratch, [&](int r) { return (rs[r].flags & kRowGeneral) != 0; });
+    if (threadIdx.x < kStreamThreads / 32) sh_n[threadIdx.x] = 0;
+    __syncthreads();
+    const WarpStage st = warp_stage(sh_buf, sh_n);
     u64 total = (u64)nF * tpr;
     int cur = -1, row = 0;
     u64 lo = 0;
@@ -441,14 +493,16 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
         int li = (int)(t / tpr);
         u32 tile = (u32)(t - (u64)li * tpr);
         if (li != cur) {
+            if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
             cur = li;
             row = sh_list[li];
             g = row_geom(x, row, d);
             lo = rs[row].lo;
         }
         if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile(g, tile, lo, rs + row, cand + (size_t)row * cap, cap);
+        filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
     }
+    if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
 }
 
 // ---------------------------------------------------------------------------
