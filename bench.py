@@ -160,6 +160,7 @@ def main():
     ap.add_argument("--config", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=0, help="override the number of workers N (smaller case for profiling)")
+    ap.add_argument("--d", type=int, default=0, help="override the vector length d (smaller case for profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -185,7 +186,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     warmup = max(args.warmup, 3)
-    wl = W.workload(args.config, N=args.rows or None)
+    wl = W.workload(args.config, d=args.d or None, N=args.rows or None)
     K_down = wl.K_down[0]
     p = W.make_p(wl)
     ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p)

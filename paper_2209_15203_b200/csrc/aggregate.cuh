@@ -2,8 +2,9 @@
 // worker order so that the fp32 result does not depend on scheduling.
 //
 // The dense server buffer (one 32-bit word per coordinate, all zero between
-// steps) is the scatter target: agg_link threads every uplink entry onto a
-// per-coordinate chain headed in that buffer; agg_reduce lets the entry at the
+// steps) is the scatter target: the uplink selection, as it emits entry number
+// e = q*K_up + slot with coordinate j, threads it onto j's chain
+// (next[e] = exchange(head[j], e+1), see emit_entry); agg_reduce lets the entry at the
 // head of each chain walk it in ascending worker order, accumulate
 //        g_j = fl(g_j + fl(p_q * v_{q,j}))        starting from +0,
 // append (j, g_j) to the union list U, put the word back to zero, and — in
@@ -15,15 +16,6 @@
 #include "common.cuh"
 
 namespace tk {
-
-__global__ void __launch_bounds__(256)
-agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, Ctrl* ctrl, u32 d) {
-    u32 e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= total) return;
-    u32 j = up[e].x;
-    if (j >= d) { raise_status(ctrl, -5); next[e] = 0; return; }
-    next[e] = atomicExch(&head[j], e + 1);
-}
 
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
@@ -56,16 +48,11 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
     }
     u32 bits = __float_as_uint(acc);
-    warp_append(owner, j, bits, &uni->cand_count, U, ucap);
-}
-
-// Start-of-step reset of the union's state and the downlink counter.
-__global__ void reset_union_kernel(RowState* uni) {
-    uni->lo = 0;
-    uni->cand_count = 0;
-    uni->max_key = 0;
-    uni->out_count = 0;
-    uni->flags = 0;
+    u32 m = warp_append(owner, j, bits, &uni->cand_count, U, ucap);
+    if (m) {  // the downlink selection wants the largest aggregated magnitude
+        u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
+        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&uni->max_key, wm);
+    }
 }
 
 // ---- helpers of the inspection calls (not on the per-step path) ----

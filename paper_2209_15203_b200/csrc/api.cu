@@ -227,7 +227,7 @@ int cluster_size_for(int64_t entries) {
     } while (0)
 
 int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, size_t list_stride, u32 cap,
-                  RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, Ctrl* ctrl) {
+                  RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(rows * cs), 1, 1);
     cfg.blockDim = dim3(kSelectThreads, 1, 1);
@@ -240,7 +240,7 @@ int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, siz
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, select_kernel, lists, list_stride, cap, rs, K, out, out_stride, apply, ctrl) !=
+    if (cudaLaunchKernelEx(&cfg, select_kernel, lists, list_stride, cap, rs, K, out, out_stride, apply, link, ctrl) !=
         cudaSuccess) {
         cudaGetLastError();
         return TK_ERR_CUDA;
@@ -251,19 +251,25 @@ int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, siz
 // Exact Top_K of every row of x into b.out ([rows][K], arbitrary order).  ev0/ev1, when
 // given, bracket the streaming pass.  *launches is advanced by the kernels enqueued.
 int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
-               Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches) {
+               Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches,
+               RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0}) {
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
     const bool predict = !force_general && d >= 262144 && K * 64 <= d;
-    int spt = 1;
-    u32 groups = 0, rank = 0;
+    int turns = 1;
+    u64 stride_fp = 0;
+    u32 rank = 0;
     if (predict) {
-        int64_t want = (d + 1024 * K - 1) / (1024 * K);
-        int64_t lim = d / 262144 < 16 ? d / 262144 : 16;
-        spt = (int)(want < 1 ? 1 : (want > lim ? lim : want));
-        groups = (u32)kSampleSlots * (u32)spt;
-        double ks = (double)K * 8.0 * groups / (double)d;  // expected top-K members in the sample
+        // sample ~32*d/K values per row (about 32 members of the top K), as whole 128-byte lines
+        const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
+        int64_t want = (32 * (d / K) + per_turn - 1) / per_turn;
+        int64_t lim = d / (8 * per_turn) < kPredictMaxTurns ? d / (8 * per_turn) : kPredictMaxTurns;
+        turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
+        if (turns < 1) turns = 1;
+        u64 lines = (u64)turns * (2 * kSampleSlots / 8);
+        stride_fp = ((u64)(d - 32) << 32) / (lines - 1);                  // run g starts near g*(d-32)/(lines-1)
+        double ks = (double)K * 32.0 * (double)lines / (double)d;          // expected top-K members in the sample
         double r = ceil(ks + 6.0 * sqrt(ks) + 4.0);
         rank = (u32)(r > kSampleSlots / 2 ? kSampleSlots / 2 : r);
     }
@@ -276,7 +282,8 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         uint2* cand = b.cand + (size_t)r0 * b.cap;
         uint2* out = b.out + (size_t)r0 * (size_t)K;
         if (predict) {
-            predict_kernel<<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, spt, groups, rank, rs, smax);
+            predict_kernel<<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs,
+                                                                                   smax, r0 == 0 ? also_reset : nullptr);
             TK_LAUNCH_CHECK();
             if (ev0) cudaEventRecord(ev0, stream);
             u64 tiles = (u64)nr * b.tpr;
@@ -287,7 +294,7 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             if (ev1) cudaEventRecord(ev1, stream);
             *launches += 2;
         } else {
-            reset_rows_kernel<<<(nr + 255) / 256, 256, 0, stream>>>(rs, nr);
+            reset_rows_kernel<<<(nr + 255) / 256, 256, 0, stream>>>(rs, nr, r0 == 0 ? also_reset : nullptr);
             TK_LAUNCH_CHECK();
             *launches += 1;
         }
@@ -304,8 +311,10 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         }
         ApplyArgs none = {nullptr, 0.0f};
         int64_t expect = predict ? 3 * K : (int64_t)b.cap;
+        LinkArgs lk = link;
+        lk.row_base = (u32)r0;
         rc = launch_select(stream, nr, cluster_size_for(expect), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, none,
-                           ctrl);
+                           lk, ctrl);
         if (rc != TK_OK) return rc;
         *launches += 1;
     }
@@ -408,29 +417,29 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     if (!c || !aligned4(w_dev) || !aligned4(grads_dev) || !isfinite(alpha)) return TK_ERR_INVALID;
     if (mode != TK_MODE_UNI && mode != TK_MODE_BIDIR) return TK_ERR_INVALID;
     cudaStream_t s = c->stream;
-    reset_union_kernel<<<1, 1, 0, s>>>(c->uni);
-    TK_LAUNCH_CHECK();
-    c->launches += 1;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
         e0 = c->ev[2 * c->ev_used];
         e1 = c->ev[2 * c->ev_used + 1];
         c->ev_used += 1;
     }
+    // the first kernel of the selection also resets the state of the union / downlink selection
+    // ... and its last kernel threads every uplink entry onto its coordinate's chain
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0};
     int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
-                        &c->launches);
+                        &c->launches, c->uni, link);
     if (rc != TK_OK) return rc;
     u32 total = (u32)(c->N * c->K_up);
     u32 blocks = (total + 255) / 256;
-    agg_link_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, c->head, c->next, c->ctrl, (u32)c->d);
-    TK_LAUNCH_CHECK();
     agg_reduce_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->uni, c->U,
                                              c->ucap, w_dev, alpha, mode == TK_MODE_UNI ? 1 : 0, c->ctrl, (u32)c->d);
     TK_LAUNCH_CHECK();
-    c->launches += 2;
+    c->launches += 1;
     if (mode == TK_MODE_BIDIR) {
         ApplyArgs ap = {w_dev, alpha};
-        rc = launch_select(s, 1, 8, c->U, c->ucap, c->ucap, c->uni, (u32)c->K_down, c->sel, c->ucap, ap, c->ctrl);
+        LinkArgs nolink = {nullptr, nullptr, 0, 0};
+        rc = launch_select(s, 1, 8, c->U, c->ucap, c->ucap, c->uni, (u32)c->K_down, c->sel, c->ucap, ap, nolink,
+                           c->ctrl);
         if (rc != TK_OK) return rc;
         c->launches += 1;
     }

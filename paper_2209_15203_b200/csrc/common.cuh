@@ -23,8 +23,9 @@ typedef unsigned long long u64;
 
 constexpr int kHistBins = 2048;        // buckets of one refinement level
 constexpr int kPredictCtas = 8;        // sampling CTAs per row
-constexpr int kPredictThreads = 512;
-constexpr int kSampleSlots = kPredictCtas * kPredictThreads;  // per-row sample maxima
+constexpr int kPredictThreads = 1024;
+constexpr int kSampleSlots = kPredictCtas * kPredictThreads / 2;  // per-row sample maxima (one per thread pair)
+constexpr int kPredictMaxTurns = 10;   // 16-byte loads one sampling thread issues, all at once
 constexpr int kStreamThreads = 512;    // streaming kernels: threads per CTA
 constexpr int kStreamUnroll = 4;       // 16-byte loads in flight per thread
 constexpr int kStreamCtasPerSm = 2;    // filter kernel: resident CTAs per SM (grid = that x SMs)

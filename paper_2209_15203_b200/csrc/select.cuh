@@ -27,131 +27,103 @@ namespace tk {
 // ---------------------------------------------------------------------------
 // predict: sample -> lower bound
 // ---------------------------------------------------------------------------
-// Each of the kSampleSlots threads of a row reads `spt` groups of 8 consecutive
-// values spread evenly over the row and keeps the largest key it saw.  The last
-// CTA of the row to finish takes the `rank`-th largest of these maxima as the
-// bound: at least `rank` sampled values are >= it, so it is never above the
-// rank-th largest sampled value.
+// The sample of a row is `lines` runs of 32 consecutive values (one 128-byte
+// line each: DRAM delivers whole lines, so narrower runs cost the same traffic)
+// spread evenly over the row (run g starts at (g * stride_fp) >> 32, rounded
+// down to a multiple of 32).  Eight neighbouring threads share a line, 4 values
+// each; a thread issues all its `turns` loads at once (the kernel is a chain of
+// DRAM latencies otherwise).  Every pair of threads keeps the largest key it
+// saw: kSampleSlots maxima per row.  The last CTA of the row to finish takes a
+// lower bound of the `rank`-th largest maximum — exact in its leading 22 bits,
+// which costs two histogram passes instead of four — as the row's bound: at
+// least `rank` sampled values are >= it.
+__device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
+    r->lo = lo;
+    r->cand_count = 0;
+    r->max_key = 0;
+    r->out_count = 0;
+    r->flags = flags;
+    r->ticket = 0;
+    r->g_active = 0;
+}
+
 __global__ void __launch_bounds__(kPredictThreads)
-predict_kernel(const float* __restrict__ x, int64_t d, int spt, u32 groups, u32 rank,
-               RowState* rs, u32* smax) {
-    __shared__ u32 sh_hist[256];
-    __shared__ u32 sh_sel[3];
+predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank,
+               RowState* rs, u32* smax, RowState* also_reset) {
+    __shared__ u32 sh_hist[kHistBins];
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_res[2];
+    __shared__ u32 sh_ticket;
     const int row = blockIdx.y;
-    const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;
+    const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;   // 0 .. 2*kSampleSlots-1
+    if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
     const float* xr = x + (size_t)row * (size_t)d;
-    const bool vec_ok = (((uintptr_t)xr) & 15u) == 0;  // groups start at multiples of 8 elements
-    const u64 span = (u64)(d - 8), div = (u64)(groups - 1);
-    u32 mx = 0;
-    for (int k0 = 0; k0 < spt; k0 += 4) {
-        uint4 a[4], b[4];
+    const bool vec_ok = (((uintptr_t)xr) & 15u) == 0;  // runs start at multiples of 32 elements
+    constexpr u32 kLinesPerTurn = 2 * kSampleSlots / 8;
+    uint4 v[kPredictMaxTurns];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            a[u] = make_uint4(0, 0, 0, 0);
-            b[u] = make_uint4(0, 0, 0, 0);
-            if (k0 + u < spt) {
-                u64 g = (u64)t + (u64)(k0 + u) * kSampleSlots;
-                u64 e = ((g * span) / div) & ~7ull;
-                if (vec_ok) {
-                    a[u] = ld_stream(reinterpret_cast<const uint4*>(xr + e));
-                    b[u] = ld_stream(reinterpret_cast<const uint4*>(xr + e) + 1);
-                } else {
-                    a[u] = make_uint4(__float_as_uint(__ldg(xr + e)), __float_as_uint(__ldg(xr + e + 1)),
-                                      __float_as_uint(__ldg(xr + e + 2)), __float_as_uint(__ldg(xr + e + 3)));
-                    b[u] = make_uint4(__float_as_uint(__ldg(xr + e + 4)), __float_as_uint(__ldg(xr + e + 5)),
-                                      __float_as_uint(__ldg(xr + e + 6)), __float_as_uint(__ldg(xr + e + 7)));
-                }
+    for (int k = 0; k < kPredictMaxTurns; ++k) {
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (k < turns) {
+            u64 g = (u64)(t >> 3) + (u64)k * kLinesPerTurn;
+            u64 e = (((g * stride_fp) >> 32) & ~31ull) + 4u * (t & 7u);
+            if (vec_ok) {
+                v[k] = ld_stream(reinterpret_cast<const uint4*>(xr + e));
+            } else {
+                v[k] = make_uint4(__float_as_uint(__ldg(xr + e)), __float_as_uint(__ldg(xr + e + 1)),
+                                  __float_as_uint(__ldg(xr + e + 2)), __float_as_uint(__ldg(xr + e + 3)));
             }
         }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            mx = max(mx, max(max(key_of(a[u].x), key_of(a[u].y)), max(key_of(a[u].z), key_of(a[u].w))));
-            mx = max(mx, max(max(key_of(b[u].x), key_of(b[u].y)), max(key_of(b[u].z), key_of(b[u].w))));
-        }
     }
-    smax[(size_t)row * kSampleSlots + t] = mx;
+    u32 mx = 0;
+#pragma unroll
+    for (int k = 0; k < kPredictMaxTurns; ++k)
+        mx = max(mx, max(max(key_of(v[k].x), key_of(v[k].y)), max(key_of(v[k].z), key_of(v[k].w))));
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    if ((t & 1u) == 0) smax[(size_t)row * kSampleSlots + (t >> 1)] = mx;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) sh_sel[0] = atomicAdd(&rs[row].ticket, 1u);
+    if (threadIdx.x == 0) sh_ticket = atomicAdd(&rs[row].ticket, 1u);
     __syncthreads();
-    if (sh_sel[0] != kPredictCtas - 1) return;
+    if (sh_ticket != kPredictCtas - 1) return;
     __threadfence();
 
-    // last CTA of the row: rank-th largest of the kSampleSlots maxima, by radix select
+    // last CTA of the row: the rank-th largest of the kSampleSlots maxima, to 22 leading bits
+    constexpr int PER = kSampleSlots / kPredictThreads;
     const volatile u32* vm = smax + (size_t)row * kSampleSlots;
-    u32 mine[kSampleSlots / kPredictThreads];
+    u32 mine[PER];
 #pragma unroll
-    for (int i = 0; i < kSampleSlots / kPredictThreads; ++i) mine[i] = vm[threadIdx.x + i * kPredictThreads];
+    for (int i = 0; i < PER; ++i) mine[i] = vm[threadIdx.x + i * kPredictThreads];
     u32 prefix = 0, need = rank;
-    for (int pass = 0; pass < 4; ++pass) {
-        const int shift = pass < 3 ? 23 - 8 * pass : 0;
-        const int nb = pass < 3 ? 256 : 128;
-        const int hs = pass < 3 ? shift + 8 : 7;  // bits above this digit
-        if (threadIdx.x < 256) sh_hist[threadIdx.x] = 0;
-        if (threadIdx.x == 0) { sh_sel[1] = 0; sh_sel[2] = 0; }
+    for (int pass = 0; pass < 2; ++pass) {
+        const int shift = pass == 0 ? 20 : 9;           // key bits 30..20, then 19..9
+        for (int b = threadIdx.x; b < kHistBins; b += kPredictThreads) sh_hist[b] = 0;
+        if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < kSampleSlots / kPredictThreads; ++i) {
-            u32 v = mine[i];
-            if ((v >> hs) == (prefix >> hs)) atomicAdd(&sh_hist[(v >> shift) & (u32)(nb - 1)], 1u);
+        for (int i = 0; i < PER; ++i) {
+            // the maxima crowd into a few bins: one shared-memory atomic per distinct bin and warp
+            u32 val = mine[i];
+            bool ok = pass == 0 || (val >> 20) == (prefix >> 20);
+            u32 bin = (val >> shift) & (u32)(kHistBins - 1);
+            u32 peers = __match_any_sync(0xffffffffu, ok ? bin : 0xffffffffu);
+            if (ok && (int)lane_id() == __ffs(peers) - 1) atomicAdd(&sh_hist[bin], (u32)__popc(peers));
         }
         __syncthreads();
-        if (threadIdx.x < 32) {
-            // lane l owns the 8 bins nb-1-8l .. nb-8-8l (descending); bins below 0 do not exist
-            u32 lane = threadIdx.x, local = 0;
-            int top = nb - 1 - 8 * (int)lane;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) if (top - i >= 0) local += sh_hist[top - i];
-            u32 incl = local;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                u32 y = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= (u32)o) incl += y;
-            }
-            u32 total = __shfl_sync(0xffffffffu, incl, 31);
-            u32 want = need <= total ? need : total;  // fewer maxima than rank: take the smallest
-            u32 excl = incl - local;
-            if (want > 0 && excl < want && want <= incl) {
-                u32 run = excl;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (top - i >= 0) {
-                        u32 h = sh_hist[top - i];
-                        if (run < want && want <= run + h) { sh_sel[1] = (u32)(top - i); sh_sel[2] = run; }
-                        run += h;
-                    }
-                }
-            }
-        }
-        __syncthreads();
-        prefix |= sh_sel[1] << shift;
-        need -= sh_sel[2];
-        __syncthreads();
+        u32 b, above;
+        find_bucket<kHistBins / kPredictThreads>(sh_hist, kHistBins, need, sh_scratch, sh_res, &b, &above);
+        if (b == 0xffffffffu) { b = 0; above = 0; }     // cannot happen (rank <= kSampleSlots)
+        prefix |= b << shift;
+        need -= above;
     }
-    if (threadIdx.x == 0) {
-        RowState* r = rs + row;
-        r->lo = (u64)prefix << 32;
-        r->cand_count = 0;
-        r->max_key = 0;
-        r->out_count = 0;
-        r->flags = 0;
-        r->ticket = 0;
-        r->g_active = 0;
-    }
+    if (threadIdx.x == 0) reset_state(rs + row, (u64)prefix << 32, 0u);
 }
 
 // No prediction: mark every row for the multi-pass path.
-__global__ void reset_rows_kernel(RowState* rs, int rows) {
+__global__ void reset_rows_kernel(RowState* rs, int rows, RowState* also_reset) {
     int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r < rows) {
-        rs[r].lo = ~0ull;
-        rs[r].cand_count = 0;
-        rs[r].max_key = 0;
-        rs[r].out_count = 0;
-        rs[r].flags = kRowGeneral;
-        rs[r].ticket = 0;
-        rs[r].g_active = 0;
-    }
+    if (r < rows) reset_state(rs + r, ~0ull, kRowGeneral);
+    if (also_reset && r == 0) reset_state(also_reset, 0ull, 0u);
 }
 
 // ---------------------------------------------------------------------------
@@ -201,11 +173,16 @@ __device__ __forceinline__ WarpStage warp_stage(uint2* sh_buf, u32* sh_n) {
 __device__ __forceinline__ void stage_flush(const WarpStage& st, RowState* rs, uint2* cand, u32 cap) {
     u32 n = *st.n;
     if (n == 0) return;
-    u32 lane = lane_id(), base = 0;
+    u32 lane = lane_id(), base = 0, mx = 0;
     if (lane == 0) base = atomicAdd(&rs->cand_count, n);
     base = __shfl_sync(0xffffffffu, base, 0);
-    for (u32 i = lane; i < n; i += 32)
-        if (base + i < cap) cand[base + i] = st.buf[i];
+    for (u32 i = lane; i < n; i += 32) {
+        uint2 e = st.buf[i];
+        mx = max(mx, key_of(e.y));
+        if (base + i < cap) cand[base + i] = e;
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    if (lane == 0) atomicMax(&rs->max_key, mx);
     __syncwarp();
     if (lane == 0) *st.n = 0;
     __syncwarp();
@@ -387,9 +364,16 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
         u32 c = rs[r].cand_count;
         return (rs[r].flags & kRowGeneral) != 0 || c < K || c > cap;
     };
+    {
+        int any = 0;
+        for (int r = threadIdx.x; r < rows; r += blockDim.x) any |= failed(r) ? 1 : 0;
+        if (!__syncthreads_or(any)) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) ctrl->rows_general = 0;
+            return;
+        }
+    }
     int nF = build_row_list(rows, sh_list, sh_scratch, failed);
     if (blockIdx.x == 0 && threadIdx.x == 0) ctrl->rows_general = (u32)nF;
-    if (nF == 0) return;
 
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nF; i += gridDim.x * blockDim.x) {
         RowState* r = rs + sh_list[i];
@@ -509,24 +493,50 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
 // select: exact K largest composite keys among a row's candidates (one cluster per row)
 // ---------------------------------------------------------------------------
 struct ApplyArgs {
-    float* w;      // if non-NULL: w[idx] -= alpha * val for every emitted entry
+    float* w;      // if non-NULL: w[idx] -= alpha * val for every emitted entry (last worker step)
     float alpha;
+};
+
+// If head is non-NULL every emitted entry (row, slot) is also threaded onto the chain of its
+// coordinate in the dense server buffer (first half of the server step, see aggregate.cuh).
+struct LinkArgs {
+    u32* head;
+    u32* next;
+    u32 d;
+    u32 row_base;  // entry ids count rows from here (rows are processed in batches)
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
 
+__device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx, u32 bits, uint2* orow,
+                                           size_t out_stride, const ApplyArgs& apply, const LinkArgs& link,
+                                           Ctrl* ctrl) {
+    if (slot >= Keff) { raise_status(ctrl, -5); return; }
+    orow[slot] = make_uint2(idx, bits);
+    if (apply.w) {
+        float upd = __fmul_rn(apply.alpha, __uint_as_float(bits));
+        apply.w[idx] = __fsub_rn(apply.w[idx], upd);
+    }
+    if (link.head) {
+        u32 e = (link.row_base + row) * (u32)out_stride + slot;
+        if (idx < link.d) link.next[e] = atomicExch(&link.head[idx], e + 1);
+        else { link.next[e] = 0; raise_status(ctrl, -5); }
+    }
+}
+
+// lists[row] holds the row's candidates: exactly the entries with ck >= rs[row].lo, all with
+// key <= rs[row].max_key, rs[row].cand_count of them.
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
-              uint2* out, size_t out_stride, ApplyArgs apply, Ctrl* ctrl) {
-    __shared__ u32 sh_hist[kHistBins];
+              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
+    __shared__ u32 sh_hist[2][kHistBins];  // double-buffered: peers may still read level L while L+1 fills
     __shared__ u32 sh_tot[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
-    __shared__ u32 sh_max;
     cg::cluster_group cluster = cg::this_cluster();
     const u32 CS = cluster.num_blocks();
     const u32 rank = cluster.block_rank();
-    const int row = blockIdx.x / CS;
+    const u32 row = blockIdx.x / CS;
     RowState* r = rs + row;
     const u32 C = min(r->cand_count, cap);
     const u32 Keff = min(K, C);
@@ -535,62 +545,55 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     const u32 stride = CS * kSelectThreads;
     const u32 rest = first + kSelectRegs * stride;  // entries from here on are re-read every level
 
-    // this thread's entries first + k*stride, k < kSelectRegs, stay in registers
-    u32 eidx[kSelectRegs], ebits[kSelectRegs];
+    // this thread's entries first + k*stride, k < kSelectRegs, stay in registers as composite
+    // keys (0 = absent; a real entry's composite key is never 0) plus one sign bit each
+    u64 eck[kSelectRegs];
+    u32 esign = 0;
 #pragma unroll
     for (int k = 0; k < kSelectRegs; ++k) {
         u32 i = first + (u32)k * stride;
-        uint2 e = i < C ? list[i] : make_uint2(0xffffffffu, 0u);  // absent: ck = 0
-        eidx[k] = e.x;
-        ebits[k] = e.y;
+        eck[k] = 0;
+        if (i < C) {
+            uint2 e = list[i];
+            eck[k] = composite(key_of(e.y), e.x);
+            esign |= (e.y >> 31) << k;
+        }
     }
 
-    u64 T = 0;  // emit entries with ck >= T
+    u64 T = 1;  // emit entries with ck >= T (absent ones are 0)
     if (C > Keff) {
-        // the largest key bounds the range from above
-        u32 mx = 0;
-#pragma unroll
-        for (int k = 0; k < kSelectRegs; ++k) mx = max(mx, key_of(ebits[k]));
-        for (u32 i = rest; i < C; i += stride) mx = max(mx, key_of(list[i].y));
-        mx = __reduce_max_sync(0xffffffffu, mx);
-        if (threadIdx.x == 0) sh_max = 0;
-        __syncthreads();
-        if (lane_id() == 0) atomicMax(&sh_max, mx);
-        cluster.sync();
-        mx = 0;
-        for (u32 c = 0; c < CS; ++c) mx = max(mx, *cluster.map_shared_rank(&sh_max, c));
-        u64 lo = r->lo;
-        u64 hi = ((u64)mx << 32) | 0xffffffffull;
+        u64 lo = max(r->lo, 1ull);
+        u64 hi = ((u64)r->max_key << 32) | 0xffffffffull;
         if (hi < lo) hi = lo;
         u32 need = Keff;
         bool found = false;
         for (int level = 0; level < 8 && !found; ++level) {
+            u32* hist = sh_hist[level & 1];
             u64 width = hi - lo;
             int s = width ? max(0, 64 - __clzll((long long)width) - 11) : 0;
             int nb = (int)(width >> s) + 1;
-            for (int b = threadIdx.x; b < nb; b += kSelectThreads) sh_hist[b] = 0;
+            for (int b = threadIdx.x; b < nb; b += kSelectThreads) hist[b] = 0;
             if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
             __syncthreads();
 #pragma unroll
             for (int k = 0; k < kSelectRegs; ++k) {
-                u64 ck = composite(key_of(ebits[k]), eidx[k]);
-                if (ck >= lo && ck <= hi && eidx[k] != 0xffffffffu) atomicAdd(&sh_hist[(u32)((ck - lo) >> s)], 1u);
+                u64 off = eck[k] - lo;              // wraps to a huge value when eck < lo
+                if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
             for (u32 i = rest; i < C; i += stride) {
                 uint2 e = list[i];
-                u64 ck = composite(key_of(e.y), e.x);
-                if (ck >= lo && ck <= hi) atomicAdd(&sh_hist[(u32)((ck - lo) >> s)], 1u);
+                u64 off = composite(key_of(e.y), e.x) - lo;
+                if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
-            cluster.sync();
+            cluster.sync();  // all CTAs of the row have filled this level's histogram
             for (int b = threadIdx.x; b < nb; b += kSelectThreads) {
                 u32 sum = 0;
-                for (u32 c = 0; c < CS; ++c) sum += cluster.map_shared_rank(sh_hist, c)[b];
+                for (u32 c = 0; c < CS; ++c) sum += cluster.map_shared_rank(hist, c)[b];
                 sh_tot[b] = sum;
             }
             __syncthreads();
             u32 b, above;
             find_bucket<kHistBins / kSelectThreads>(sh_tot, nb, need, sh_scratch, sh_res, &b, &above);
-            cluster.sync();  // every CTA is done reading its peers' histograms
             if (b == 0xffffffffu) {
                 if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
                 break;
@@ -608,36 +611,37 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             T = lo;
             if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
         }
+        cluster.sync();  // no CTA leaves while a peer may still read its histograms
     }
 
-    // emission: every entry with ck >= T, exactly Keff of them
+    // emission: every entry with ck >= T, exactly Keff of them; one counter update per warp
     uint2* orow = out + (size_t)row * out_stride;
-    auto emit = [&](bool pred, u32 idx, u32 bits) {
-        u32 m = __ballot_sync(0xffffffffu, pred);
-        if (m == 0) return;
-        u32 lane = lane_id(), base = 0;
-        int leader = __ffs(m) - 1;
-        if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
-        base = __shfl_sync(0xffffffffu, base, leader);
-        if (pred) {
-            u32 slot = base + (u32)__popc(m & ((1u << lane) - 1u));
-            if (slot < Keff) {
-                orow[slot] = make_uint2(idx, bits);
-                if (apply.w) {
-                    float upd = __fmul_rn(apply.alpha, __uint_as_float(bits));
-                    apply.w[idx] = __fsub_rn(apply.w[idx], upd);
-                }
-            } else {
-                raise_status(ctrl, -5);
-            }
-        }
-    };
-    // counts per thread first, so that one atomic per warp covers all register-held entries
+    u32 mine = 0;
 #pragma unroll
-    for (int k = 0; k < kSelectRegs; ++k) {
-        if (__any_sync(0xffffffffu, first + (u32)k * stride < C)) {
-            bool pred = eidx[k] != 0xffffffffu && composite(key_of(ebits[k]), eidx[k]) >= T;
-            emit(pred, eidx[k], ebits[k]);
+    for (int k = 0; k < kSelectRegs; ++k) mine += eck[k] >= T ? 1u : 0u;
+    {
+        u32 lane = lane_id();
+        u32 incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            u32 y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= (u32)o) incl += y;
+        }
+        u32 wtotal = __shfl_sync(0xffffffffu, incl, 31);
+        u32 base = 0;
+        if (wtotal) {
+            if (lane == 31) base = atomicAdd(&r->out_count, wtotal);
+            base = __shfl_sync(0xffffffffu, base, 31);
+        }
+        u32 slot = base + incl - mine;
+#pragma unroll
+        for (int k = 0; k < kSelectRegs; ++k) {
+            if (eck[k] >= T) {
+                u32 idx = 0xffffffffu - (u32)eck[k];
+                u32 bits = (u32)(eck[k] >> 32) | (((esign >> k) & 1u) << 31);
+                emit_entry(row, slot, Keff, idx, bits, orow, out_stride, apply, link, ctrl);
+                ++slot;
+            }
         }
     }
     for (u32 i0 = rank * kSelectThreads + kSelectRegs * stride; i0 < C; i0 += stride) {
@@ -648,7 +652,14 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             e = list[i];
             pred = composite(key_of(e.y), e.x) >= T;
         }
-        emit(pred, e.x, e.y);
+        u32 m = __ballot_sync(0xffffffffu, pred);
+        if (m == 0) continue;
+        u32 lane = lane_id(), base = 0;
+        int leader = __ffs(m) - 1;
+        if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
+        base = __shfl_sync(0xffffffffu, base, leader);
+        if (pred) emit_entry(row, base + (u32)__popc(m & ((1u << lane) - 1u)), Keff, e.x, e.y, orow, out_stride,
+                             apply, link, ctrl);
     }
 }
 
