@@ -235,10 +235,10 @@ def main():
     # roofline of the dominant kernel (the streaming selection pass)
     peak, peak_kind = measured_hbm_gbs()
     roof = None
-    if st.select_samples > 0:
+    if st.select_samples > 0 and st.select_ms_sum > 0:
         k_ms = st.select_ms_sum / st.select_samples
         achieved = 4.0 * elems / (k_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "kernel": "filter_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        roof = {"bound": "hbm", "kernel": "filter_kernel" if st.rows_general == 0 else "general_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind, "traffic": FILTER_TRAFFIC_BYTES,
                 "algorithmic_bytes": 4 * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
 

@@ -285,13 +285,13 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             predict_kernel<<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs,
                                                                                    smax, r0 == 0 ? also_reset : nullptr);
             TK_LAUNCH_CHECK();
-            if (ev0) cudaEventRecord(ev0, stream);
+            if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             u64 tiles = (u64)nr * b.tpr;
             u64 resident = (u64)di->sms * kStreamCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
             u32 grid = (u32)(tiles < resident ? tiles : resident);
-            filter_kernel<<<grid, kStreamThreads, 0, stream>>>(xb, nr, d, b.tpr, rs, cand, b.cap);
+            filter_kernel<<<grid, kStreamThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, b.tpr, rs, cand, b.cap);
             TK_LAUNCH_CHECK();
-            if (ev1) cudaEventRecord(ev1, stream);
+            if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 2;
         } else {
             reset_rows_kernel<<<(nr + 255) / 256, 256, 0, stream>>>(rs, nr, r0 == 0 ? also_reset : nullptr);
@@ -302,11 +302,14 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             u32 Ku = (u32)K, tpr = b.tpr, cap = b.cap;
             void* args[] = {(void*)&xb, (void*)&nr, (void*)&d, (void*)&Ku, (void*)&tpr, (void*)&cap,
                             (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl};
+            // without a prediction the multi-pass kernel is the streaming pass that gets timed
+            if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kStreamThreads), args,
                                             0, stream) != cudaSuccess) {
                 cudaGetLastError();
                 return TK_ERR_CUDA;
             }
+            if (!predict && ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 1;
         }
         ApplyArgs none = {nullptr, 0.0f};

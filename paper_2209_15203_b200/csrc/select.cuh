@@ -204,38 +204,86 @@ __device__ __forceinline__ void consider(bool live, u32 idx, u32 bits, u64 lo, c
     __syncwarp();
 }
 
+// The four components of one float4 per lane, with at least one hit somewhere in the warp:
+// stage all qualifying components with a single update of the warp's fill count.
+__device__ __forceinline__ void consider4(uint4 v, u32 i0, u32 tk, u64 lo, const WarpStage& st,
+                                          RowState* rs, uint2* cand, u32 cap) {
+    bool p0 = key_of(v.x) >= tk, p1 = key_of(v.y) >= tk, p2 = key_of(v.z) >= tk, p3 = key_of(v.w) >= tk;
+    if ((u32)lo != 0u) {  // the bound reaches into the index bits (multi-pass path only): exact test
+        p0 = p0 && composite(key_of(v.x), i0 + 0) >= lo;
+        p1 = p1 && composite(key_of(v.y), i0 + 1) >= lo;
+        p2 = p2 && composite(key_of(v.z), i0 + 2) >= lo;
+        p3 = p3 && composite(key_of(v.w), i0 + 3) >= lo;
+    }
+    const u32 m0 = __ballot_sync(0xffffffffu, p0), m1 = __ballot_sync(0xffffffffu, p1);
+    const u32 m2 = __ballot_sync(0xffffffffu, p2), m3 = __ballot_sync(0xffffffffu, p3);
+    const u32 c0 = (u32)__popc(m0), c1 = (u32)__popc(m1), c2 = (u32)__popc(m2), c3 = (u32)__popc(m3);
+    const u32 cnt = c0 + c1 + c2 + c3;
+    if (cnt == 0) return;
+    if (cnt > kStageSlots) {  // more than the stage holds (needs > 16 hits per component on average)
+        consider(p0, i0 + 0, v.x, 0ull, st, rs, cand, cap);
+        consider(p1, i0 + 1, v.y, 0ull, st, rs, cand, cap);
+        consider(p2, i0 + 2, v.z, 0ull, st, rs, cand, cap);
+        consider(p3, i0 + 3, v.w, 0ull, st, rs, cand, cap);
+        return;
+    }
+    if (*st.n + cnt > kStageSlots) stage_flush(st, rs, cand, cap);
+    const u32 n = *st.n;
+    const u32 lt = (1u << lane_id()) - 1u;
+    if (p0) st.buf[n + (u32)__popc(m0 & lt)] = make_uint2(i0 + 0, v.x);
+    if (p1) st.buf[n + c0 + (u32)__popc(m1 & lt)] = make_uint2(i0 + 1, v.y);
+    if (p2) st.buf[n + c0 + c1 + (u32)__popc(m2 & lt)] = make_uint2(i0 + 2, v.z);
+    if (p3) st.buf[n + c0 + c1 + c2 + (u32)__popc(m3 & lt)] = make_uint2(i0 + 3, v.w);
+    __syncwarp();
+    if (lane_id() == 0) *st.n = n + cnt;
+    __syncwarp();
+}
+
+// Cheap per-float4 pre-test: could any of the four components have key >= tk?  Done in
+// floating point (|x| >= thr with thr = the float whose bits are tk; "not less than", so
+// that a NaN on either side passes) because the absolute value is free there.  It may
+// pass too much, never too little; the staging code repeats the test exactly on the keys.
+__device__ __forceinline__ bool may_hit(uint4 v, float thr) {
+    return !(fabsf(__uint_as_float(v.x)) < thr) || !(fabsf(__uint_as_float(v.y)) < thr) ||
+           !(fabsf(__uint_as_float(v.z)) < thr) || !(fabsf(__uint_as_float(v.w)) < thr);
+}
+
 // Process tile `tile` (kTileVecs float4) of a row.  All threads of the CTA call.
 __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
                                             RowState* rs, uint2* cand, u32 cap) {
     const u32 tk = (u32)(lo >> 32);
+    const float thr = __uint_as_float(tk);
     const u32 j0 = tile * kTileVecs + threadIdx.x;
+    const uint4* p = g.vec + j0;
     uint4 v[kStreamUnroll];
     bool inb[kStreamUnroll];
-    const bool full = (u64)(tile + 1) * kTileVecs <= (u64)g.nv;
+    const bool full = (tile + 1) * (u32)kTileVecs <= g.nv;
     if (full) {
 #pragma unroll
         for (int u = 0; u < kStreamUnroll; ++u) {
-            v[u] = ld_stream(g.vec + j0 + u * kStreamThreads);
+            v[u] = ld_stream(p + u * kStreamThreads);
             inb[u] = true;
         }
     } else {
 #pragma unroll
         for (int u = 0; u < kStreamUnroll; ++u) {
-            u32 j = j0 + u * kStreamThreads;
-            inb[u] = j < g.nv;
-            v[u] = inb[u] ? ld_stream(g.vec + j) : make_uint4(0, 0, 0, 0);
+            inb[u] = j0 + u * kStreamThreads < g.nv;
+            v[u] = inb[u] ? ld_stream(p + u * kStreamThreads) : make_uint4(0, 0, 0, 0);
         }
     }
 #pragma unroll
     for (int u = 0; u < kStreamUnroll; ++u) {
-        u32 m = max(max(key_of(v[u].x), key_of(v[u].y)), max(key_of(v[u].z), key_of(v[u].w)));
-        bool hit = inb[u] && m >= tk;
+        bool hit = inb[u] && may_hit(v[u], thr);
         if (__any_sync(0xffffffffu, hit)) {
             u32 i0 = g.head + 4u * (j0 + u * kStreamThreads);
-            consider(hit && key_of(v[u].x) >= tk, i0 + 0, v[u].x, lo, st, rs, cand, cap);
-            consider(hit && key_of(v[u].y) >= tk, i0 + 1, v[u].y, lo, st, rs, cand, cap);
-            consider(hit && key_of(v[u].z) >= tk, i0 + 2, v[u].z, lo, st, rs, cand, cap);
-            consider(hit && key_of(v[u].w) >= tk, i0 + 3, v[u].w, lo, st, rs, cand, cap);
+            if (tk == 0) {  // everything in the row qualifies; only the padding lanes must stay out
+                consider(hit, i0 + 0, v[u].x, lo, st, rs, cand, cap);
+                consider(hit, i0 + 1, v[u].y, lo, st, rs, cand, cap);
+                consider(hit, i0 + 2, v[u].z, lo, st, rs, cand, cap);
+                consider(hit, i0 + 3, v[u].w, lo, st, rs, cand, cap);
+            } else {        // padding lanes hold zeros, whose key is below tk
+                consider4(v[u], i0, tk, lo, st, rs, cand, cap);
+            }
         }
     }
     if (tile == 0 && threadIdx.x < 32 && (g.head | g.tail)) {
@@ -252,8 +300,10 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
 __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowState* rs,
               uint2* cand, u32 cap) {
+    extern __shared__ u64 sh_lo[];  // every row's bound, fetched once: a CTA visits all rows
     __shared__ uint2 sh_buf[(kStreamThreads / 32) * kStageSlots];
     __shared__ u32 sh_n[kStreamThreads / 32];
+    for (int r = threadIdx.x; r < rows; r += kStreamThreads) sh_lo[r] = rs[r].lo;
     if (threadIdx.x < kStreamThreads / 32) sh_n[threadIdx.x] = 0;
     __syncthreads();
     const WarpStage st = warp_stage(sh_buf, sh_n);
@@ -261,17 +311,19 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowStat
     int cur = -1;
     RowGeom g;
     u64 lo = 0;
+    int row = (int)(blockIdx.x / tpr);
+    u32 tile = blockIdx.x - (u32)row * tpr;
     for (u32 t = blockIdx.x; t < total; t += gridDim.x) {
-        int row = (int)(t / tpr);
-        u32 tile = t - (u32)row * tpr;
         if (row != cur) {
             if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
             cur = row;
             g = row_geom(x, row, d);
-            lo = rs[row].lo;
+            lo = sh_lo[row];
         }
-        if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        if (tile * (u32)kTileVecs < g.nv || tile == 0)
+            filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        tile += gridDim.x;
+        while (tile >= tpr) { tile -= tpr; ++row; }
     }
     if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
 }
