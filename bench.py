@@ -175,7 +175,7 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2209_15203_b200 import binding
+    from paper_2209_15203_b200 import binding, replicas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -198,8 +198,7 @@ def main():
     mode = binding.TK_MODE_BIDIR
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for s in range(warmup):
@@ -224,12 +223,8 @@ def main():
     sampler.join(timeout=2.0)
     ctx.tk_set_profile(False)
 
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
     elems = wl.N * wl.d
-    value = world * elems * args.steps / (ms_max * 1e-3)
+    value, ms_max = replicas.whole_job_throughput(ms, elems, args.steps, dev)
     ms_per_step = ms_max / args.steps
 
     # roofline of the dominant kernel (the streaming selection pass)
@@ -257,12 +252,10 @@ def main():
             ctx.tk_step_host(w_host, g_host, wl.alpha, mode)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * elems * n_e2e / float(tt.item()), "unit": UNIT,
+        e2e_value, e2e_ms = replicas.whole_job_throughput(dt * 1e3, elems, n_e2e, dev)
+        e2e = {"value": e2e_value, "unit": UNIT,
                "h2d_bytes_per_step": 4 * (elems + wl.d), "d2h_bytes_per_step": 4 * wl.d, "steps": n_e2e,
-               "ms_per_step": 1e3 * float(tt.item()) / n_e2e}
+               "ms_per_step": e2e_ms / n_e2e}
         del g_host, w_host
 
     # the CPU oracle on this host's cores: one full step of the same workload (rank 0, single GPU only)

@@ -36,7 +36,7 @@ int device_info(DeviceInfo** out) {
         int coop = 0, per_sm = 0;
         if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TK_ERR_CUDA;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return TK_ERR_CUDA;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, general_kernel, kStreamThreads, 0) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, general_kernel, kGeneralThreads, 0) != cudaSuccess ||
             per_sm < 1)
             return TK_ERR_CUDA;
         di.general_grid = per_sm * di.sms;
@@ -54,12 +54,13 @@ struct SelectBufs {
     uint2* cand = nullptr;    // [rows][cap]
     uint2* out = nullptr;     // [rows][K]
     u32 cap = 0;
-    u32 tpr = 0;              // tiles per row
+    u32 tpr_filter = 0;       // tiles per row of the filter kernel / of the multi-pass kernel
+    u32 tpr_general = 0;
 };
 
 struct SelectLayout {
     size_t off_rs, off_hist, off_smax, off_cand, off_out, bytes;
-    u32 cap, tpr;
+    u32 cap, tpr_filter, tpr_general;
 };
 
 u32 candidate_capacity(int64_t d, int64_t K) {
@@ -72,8 +73,9 @@ SelectLayout select_layout(int64_t rows, int64_t d, int64_t K) {
     SelectLayout L;
     L.cap = candidate_capacity(d, K);
     int64_t nv = (d + 3) / 4;
-    int64_t tpr = (nv + kTileVecs - 1) / kTileVecs;
-    L.tpr = (u32)(tpr < 1 ? 1 : tpr);
+    int64_t tf = (nv + kFilterTileVecs - 1) / kFilterTileVecs, tg = (nv + kGeneralTileVecs - 1) / kGeneralTileVecs;
+    L.tpr_filter = (u32)(tf < 1 ? 1 : tf);
+    L.tpr_general = (u32)(tg < 1 ? 1 : tg);
     size_t o = 0;
     L.off_rs = o;   o += align_up((size_t)rows * sizeof(RowState));
     L.off_hist = o; o += align_up((size_t)rows * kHistBins * sizeof(u32));
@@ -92,7 +94,8 @@ SelectBufs bind(const SelectLayout& L, char* base) {
     b.cand = (uint2*)(base + L.off_cand);
     b.out = (uint2*)(base + L.off_out);
     b.cap = L.cap;
-    b.tpr = L.tpr;
+    b.tpr_filter = L.tpr_filter;
+    b.tpr_general = L.tpr_general;
     return b;
 }
 
@@ -261,9 +264,10 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
     u64 stride_fp = 0;
     u32 rank = 0;
     if (predict) {
-        // sample ~32*d/K values per row (about 32 members of the top K), as whole 128-byte lines
+        // sample ~128*d/K values per row (about 128 members of the top K; fewer when that would take
+        // more than kPredictMaxTurns loads per thread), as whole 128-byte lines
         const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
-        int64_t want = (32 * (d / K) + per_turn - 1) / per_turn;
+        int64_t want = (128 * (d / K) + per_turn - 1) / per_turn;
         int64_t lim = d / (8 * per_turn) < kPredictMaxTurns ? d / (8 * per_turn) : kPredictMaxTurns;
         turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
         if (turns < 1) turns = 1;
@@ -286,10 +290,14 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
                                                                                    smax, r0 == 0 ? also_reset : nullptr);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
-            u64 tiles = (u64)nr * b.tpr;
-            u64 resident = (u64)di->sms * kStreamCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
+            u64 tiles = (u64)nr * b.tpr_filter;
+            u64 resident = (u64)di->sms * kFilterCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
             u32 grid = (u32)(tiles < resident ? tiles : resident);
-            filter_kernel<<<grid, kStreamThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, b.tpr, rs, cand, b.cap);
+            u32 parts = 1;
+            if (tiles >= 4 * resident) parts = (u32)(nr < kFilterPartitions ? nr : kFilterPartitions);
+            u32 cpp = grid / parts;
+            filter_kernel<<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, b.tpr_filter, parts, cpp,
+                                                                                        rs, cand, b.cap);
             TK_LAUNCH_CHECK();
             if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 2;
@@ -299,12 +307,12 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             *launches += 1;
         }
         {
-            u32 Ku = (u32)K, tpr = b.tpr, cap = b.cap;
+            u32 Ku = (u32)K, tpr = b.tpr_general, cap = b.cap;
             void* args[] = {(void*)&xb, (void*)&nr, (void*)&d, (void*)&Ku, (void*)&tpr, (void*)&cap,
                             (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl};
             // without a prediction the multi-pass kernel is the streaming pass that gets timed
             if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
-            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kStreamThreads), args,
+            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kGeneralThreads), args,
                                             0, stream) != cudaSuccess) {
                 cudaGetLastError();
                 return TK_ERR_CUDA;

@@ -26,10 +26,26 @@ constexpr int kPredictCtas = 8;        // sampling CTAs per row
 constexpr int kPredictThreads = 1024;
 constexpr int kSampleSlots = kPredictCtas * kPredictThreads / 2;  // per-row sample maxima (one per thread pair)
 constexpr int kPredictMaxTurns = 10;   // 16-byte loads one sampling thread issues, all at once
-constexpr int kStreamThreads = 512;    // streaming kernels: threads per CTA
-constexpr int kStreamUnroll = 4;       // 16-byte loads in flight per thread
-constexpr int kStreamCtasPerSm = 2;    // filter kernel: resident CTAs per SM (grid = that x SMs)
-constexpr int kTileVecs = kStreamThreads * kStreamUnroll;     // float4 per tile
+// Streaming passes.  Measured on B200: read bandwidth peaks with about 900-1150 threads and
+// 65-80 KB of loads in flight per SM and falls off sharply on either side (more resident
+// threads or deeper unrolling lose 20 %), so the filter kernel runs 2 CTAs of 448 threads
+// per SM with 5 x 16 bytes in flight per thread, as one wave.
+#ifndef TK_FILTER_THREADS
+#define TK_FILTER_THREADS 448
+#endif
+#ifndef TK_FILTER_CTAS
+#define TK_FILTER_CTAS 2
+#endif
+#ifndef TK_STREAM_UNROLL
+#define TK_STREAM_UNROLL 5
+#endif
+constexpr int kFilterThreads = TK_FILTER_THREADS;  // filter kernel: threads per CTA
+constexpr int kFilterCtasPerSm = TK_FILTER_CTAS;   // filter kernel: resident CTAs per SM (grid = that x SMs)
+constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads per CTA
+constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
+constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
+constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
+constexpr int kFilterPartitions = 8;   // the filter grid splits the tile space into this many ranges
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path

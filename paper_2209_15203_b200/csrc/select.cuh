@@ -244,38 +244,40 @@ __device__ __forceinline__ void consider4(uint4 v, u32 i0, u32 tk, u64 lo, const
 // that a NaN on either side passes) because the absolute value is free there.  It may
 // pass too much, never too little; the staging code repeats the test exactly on the keys.
 __device__ __forceinline__ bool may_hit(uint4 v, float thr) {
-    return !(fabsf(__uint_as_float(v.x)) < thr) || !(fabsf(__uint_as_float(v.y)) < thr) ||
-           !(fabsf(__uint_as_float(v.z)) < thr) || !(fabsf(__uint_as_float(v.w)) < thr);
+    // bitwise, not short-circuit: four compares and no branches
+    return (!(fabsf(__uint_as_float(v.x)) < thr)) | (!(fabsf(__uint_as_float(v.y)) < thr)) |
+           (!(fabsf(__uint_as_float(v.z)) < thr)) | (!(fabsf(__uint_as_float(v.w)) < thr));
 }
 
-// Process tile `tile` (kTileVecs float4) of a row.  All threads of the CTA call.
+// Process tile `tile` (THREADS * kStreamUnroll float4) of a row.  All THREADS threads of the CTA call.
+template <int THREADS>
 __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
                                             RowState* rs, uint2* cand, u32 cap) {
     const u32 tk = (u32)(lo >> 32);
     const float thr = __uint_as_float(tk);
-    const u32 j0 = tile * kTileVecs + threadIdx.x;
+    const u32 j0 = tile * (THREADS * kStreamUnroll) + threadIdx.x;
     const uint4* p = g.vec + j0;
     uint4 v[kStreamUnroll];
     bool inb[kStreamUnroll];
-    const bool full = (tile + 1) * (u32)kTileVecs <= g.nv;
+    const bool full = (tile + 1) * (u32)(THREADS * kStreamUnroll) <= g.nv;
     if (full) {
 #pragma unroll
         for (int u = 0; u < kStreamUnroll; ++u) {
-            v[u] = ld_stream(p + u * kStreamThreads);
+            v[u] = ld_stream(p + u * THREADS);
             inb[u] = true;
         }
     } else {
 #pragma unroll
         for (int u = 0; u < kStreamUnroll; ++u) {
-            inb[u] = j0 + u * kStreamThreads < g.nv;
-            v[u] = inb[u] ? ld_stream(p + u * kStreamThreads) : make_uint4(0, 0, 0, 0);
+            inb[u] = j0 + u * THREADS < g.nv;
+            v[u] = inb[u] ? ld_stream(p + u * THREADS) : make_uint4(0, 0, 0, 0);
         }
     }
 #pragma unroll
     for (int u = 0; u < kStreamUnroll; ++u) {
         bool hit = inb[u] && may_hit(v[u], thr);
         if (__any_sync(0xffffffffu, hit)) {
-            u32 i0 = g.head + 4u * (j0 + u * kStreamThreads);
+            u32 i0 = g.head + 4u * (j0 + u * THREADS);
             if (tk == 0) {  // everything in the row qualifies; only the padding lanes must stay out
                 consider(hit, i0 + 0, v[u].x, lo, st, rs, cand, cap);
                 consider(hit, i0 + 1, v[u].y, lo, st, rs, cand, cap);
@@ -297,32 +299,41 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
     }
 }
 
-__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
-filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, RowState* rs,
-              uint2* cand, u32 cap) {
-    extern __shared__ u64 sh_lo[];  // every row's bound, fetched once: a CTA visits all rows
-    __shared__ uint2 sh_buf[(kStreamThreads / 32) * kStageSlots];
-    __shared__ u32 sh_n[kStreamThreads / 32];
-    for (int r = threadIdx.x; r < rows; r += kStreamThreads) sh_lo[r] = rs[r].lo;
-    if (threadIdx.x < kStreamThreads / 32) sh_n[threadIdx.x] = 0;
+// The tile space (row-major: all tiles of row 0, then row 1, ...) is cut into `parts`
+// equal contiguous ranges; `cpp` CTAs share a range and interleave its tiles.  With one
+// range every CTA would visit every row, and each change of row costs a flush of the
+// staged candidates (a global atomic round trip); with one range per CTA a CTA that
+// lands in a layer full of candidates would finish late.
+__global__ void __launch_bounds__(kFilterThreads, kFilterCtasPerSm)
+filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 parts, u32 cpp,
+              RowState* rs, uint2* cand, u32 cap) {
+    extern __shared__ u64 sh_lo[];  // every row's bound, fetched once
+    __shared__ uint2 sh_buf[(kFilterThreads / 32) * kStageSlots];
+    __shared__ u32 sh_n[kFilterThreads / 32];
+    const u32 part = blockIdx.x / cpp;
+    if (part >= parts) return;
+    for (int r = threadIdx.x; r < rows; r += kFilterThreads) sh_lo[r] = rs[r].lo;
+    if (threadIdx.x < kFilterThreads / 32) sh_n[threadIdx.x] = 0;
     __syncthreads();
     const WarpStage st = warp_stage(sh_buf, sh_n);
-    const u32 total = (u32)rows * tpr;
+    const u64 total = (u64)rows * tpr;
+    const u64 t_end = (u64)(part + 1) * total / parts;
+    u64 t = (u64)part * total / parts + (blockIdx.x - part * cpp);
     int cur = -1;
     RowGeom g;
     u64 lo = 0;
-    int row = (int)(blockIdx.x / tpr);
-    u32 tile = blockIdx.x - (u32)row * tpr;
-    for (u32 t = blockIdx.x; t < total; t += gridDim.x) {
+    int row = (int)(t / tpr);
+    u32 tile = (u32)(t - (u64)row * tpr);
+    for (; t < t_end; t += cpp) {
         if (row != cur) {
             if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
             cur = row;
             g = row_geom(x, row, d);
             lo = sh_lo[row];
         }
-        if (tile * (u32)kTileVecs < g.nv || tile == 0)
-            filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
-        tile += gridDim.x;
+        if (tile * (u32)kFilterTileVecs < g.nv || tile == 0)
+            filter_tile<kFilterThreads>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        tile += cpp;
         while (tile >= tpr) { tile -= tpr; ++row; }
     }
     if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
@@ -355,10 +366,10 @@ __device__ __forceinline__ void hist_component(bool live, u32 idx, u32 bits, int
 __device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level, u64 lo,
                                           u32* sh_hist) {
     const int shift = kLevelShift[level], nbits = kLevelBits[level];
-    const u32 j0 = tile * kTileVecs + threadIdx.x;
+    const u32 j0 = tile * kGeneralTileVecs + threadIdx.x;
 #pragma unroll
     for (int u = 0; u < kStreamUnroll; ++u) {
-        u32 j = j0 + u * kStreamThreads;
+        u32 j = j0 + u * kGeneralThreads;
         if (j < g.nv) {
             uint4 v = ld_stream(g.vec + j);
             u32 i0 = g.head + 4u * j;
@@ -383,7 +394,7 @@ __device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level,
 template <typename Pred>
 __device__ __forceinline__ int build_row_list(int rows, unsigned short* sh_list, u32* scratch,
                                               Pred pred) {
-    constexpr int PER = kMaxRowsPerLaunch / kStreamThreads;
+    constexpr int PER = kMaxRowsPerLaunch / kGeneralThreads;
     u32 flags = 0, cnt = 0;
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
@@ -399,15 +410,15 @@ __device__ __forceinline__ int build_row_list(int rows, unsigned short* sh_list,
     return (int)total;
 }
 
-__global__ void __launch_bounds__(kStreamThreads)
+__global__ void __launch_bounds__(kGeneralThreads)
 general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr, u32 cap,
                RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ unsigned short sh_list[kMaxRowsPerLaunch];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
-    __shared__ uint2 sh_buf[(kStreamThreads / 32) * kStageSlots];
-    __shared__ u32 sh_n[kStreamThreads / 32];
+    __shared__ uint2 sh_buf[(kGeneralThreads / 32) * kStageSlots];
+    __shared__ u32 sh_n[kGeneralThreads / 32];
     cg::grid_group grid = cg::this_grid();
 
     // Which rows failed verification?  Nothing below modifies a RowState before
@@ -466,7 +477,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
                     for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
                     __syncthreads();
                 }
-                if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
+                if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
                 hist_tile(g, tile, level, lo, sh_hist);
             }
             if (cur >= 0) {
@@ -491,7 +502,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
             if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
             __syncthreads();
             u32 need = r->g_need, b, above;
-            find_bucket<kHistBins / kStreamThreads>(sh_hist, nb, need, sh_scratch, sh_res, &b, &above);
+            find_bucket<kHistBins / kGeneralThreads>(sh_hist, nb, need, sh_scratch, sh_res, &b, &above);
             if (threadIdx.x == 0) {
                 if (b == 0xffffffffu) {           // the row holds fewer than `need` entries: cannot happen
                     raise_status(ctrl, -5);
@@ -518,7 +529,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
 
     // phase C: filter the failed rows again with their exact bound
     nF = build_row_list(rows, sh_list, sh_scratch, [&](int r) { return (rs[r].flags & kRowGeneral) != 0; });
-    if (threadIdx.x < kStreamThreads / 32) sh_n[threadIdx.x] = 0;
+    if (threadIdx.x < kGeneralThreads / 32) sh_n[threadIdx.x] = 0;
     __syncthreads();
     const WarpStage st = warp_stage(sh_buf, sh_n);
     u64 total = (u64)nF * tpr;
@@ -535,8 +546,8 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
             g = row_geom(x, row, d);
             lo = rs[row].lo;
         }
-        if ((u64)tile * kTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
+        filter_tile<kGeneralThreads>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
     }
     if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
 }
