@@ -25,6 +25,7 @@ struct DeviceInfo {
     bool ready = false;
     int sms = 0;
     int general_grid = 0;  // co-resident CTAs of general_kernel
+    int select_grid = 0;   // co-resident CTAs of the grid-wide select_kernel
 };
 DeviceInfo g_dev[64];
 
@@ -40,6 +41,10 @@ int device_info(DeviceInfo** out) {
             per_sm < 1)
             return TK_ERR_CUDA;
         di.general_grid = per_sm * di.sms;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel<true>, kSelectThreads, 0) != cudaSuccess ||
+            per_sm < 1)
+            return TK_ERR_CUDA;
+        di.select_grid = per_sm * di.sms;
         di.ready = true;
     }
     *out = &di;
@@ -172,6 +177,7 @@ struct tk_ctx {
     u32* next = nullptr;       // [N*K_up]
     uint2* U = nullptr;        // [ucap] aggregate over the union
     uint2* sel = nullptr;      // [ucap] downlink message (unordered)
+    u32* ghist = nullptr;      // [3][kHistBins] histograms of the grid-wide select, zero at rest
     u32 ucap = 0;
     // host state
     int force_general = 0;
@@ -189,7 +195,7 @@ struct tk_ctx {
 namespace {
 
 struct CtxLayout {
-    size_t off_ctrl, off_p, off_sel_up, off_uni, off_head, off_next, off_U, off_sel, bytes;
+    size_t off_ctrl, off_p, off_sel_up, off_uni, off_head, off_next, off_U, off_sel, off_ghist, bytes;
     SelectLayout up;
     u32 ucap;
 };
@@ -213,6 +219,7 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
     L.off_next = o;   o += align_up((size_t)(N * K_up) * sizeof(u32));
     L.off_U = o;      o += align_up((size_t)ucap * sizeof(uint2));
     L.off_sel = o;    o += align_up((size_t)ucap * sizeof(uint2));
+    L.off_ghist = o;  o += align_up((size_t)3 * kHistBins * sizeof(u32));
     L.bytes = o;
     return L;
 }
@@ -243,7 +250,24 @@ int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, siz
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, select_kernel, lists, list_stride, cap, rs, K, out, out_stride, apply, link, ctrl) !=
+    u32* no_ghist = nullptr;
+    if (cudaLaunchKernelEx(&cfg, select_kernel<false>, lists, list_stride, cap, rs, K, out, out_stride, apply, link, ctrl,
+                           no_ghist) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return TK_OK;
+}
+
+// One long list selected by the whole grid (cooperative launch).
+int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap, RowState* rs, u32 K, uint2* out,
+                       ApplyArgs apply, Ctrl* ctrl, u32* ghist) {
+    size_t stride = cap;
+    LinkArgs nolink = {nullptr, nullptr, 0, 0};
+    void* args[] = {(void*)&list, (void*)&stride, (void*)&cap, (void*)&rs,  (void*)&K,    (void*)&out,
+                    (void*)&stride, (void*)&apply, (void*)&nolink, (void*)&ctrl, (void*)&ghist};
+    if (cudaLaunchCooperativeKernel((void*)select_kernel<true>, dim3(ctas), dim3(kSelectThreads), args, 0, stream) !=
         cudaSuccess) {
         cudaGetLastError();
         return TK_ERR_CUDA;
@@ -405,12 +429,14 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
     c->next = (u32*)(c->ws + L.off_next);
     c->U = (uint2*)(c->ws + L.off_U);
     c->sel = (uint2*)(c->ws + L.off_sel);
+    c->ghist = (u32*)(c->ws + L.off_ghist);
     c->ucap = L.ucap;
     // state that must be zero at rest: control block, row states, histograms, the dense buffer
     bool ok = cudaMemsetAsync(c->ctrl, 0, sizeof(Ctrl), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->up.rs, 0, (size_t)N * sizeof(RowState), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->up.hist, 0, (size_t)N * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->uni, 0, sizeof(RowState), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->ghist, 0, (size_t)3 * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->head, 0, (size_t)d * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemcpyAsync(c->p, p_host, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream) ==
                   cudaSuccess &&
@@ -448,9 +474,14 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     c->launches += 1;
     if (mode == TK_MODE_BIDIR) {
         ApplyArgs ap = {w_dev, alpha};
-        LinkArgs nolink = {nullptr, nullptr, 0, 0};
-        rc = launch_select(s, 1, 8, c->U, c->ucap, c->ucap, c->uni, (u32)c->K_down, c->sel, c->ucap, ap, nolink,
-                           c->ctrl);
+        DeviceInfo* di = nullptr;
+        rc = device_info(&di);
+        if (rc != TK_OK) return rc;
+        // the union can hold up to ucap entries: about 4096 per CTA, at most one co-resident wave
+        int ctas = (int)((c->ucap + 4095) / 4096);
+        if (ctas > di->select_grid) ctas = di->select_grid;
+        if (ctas < 1) ctas = 1;
+        rc = launch_select_grid(s, ctas, c->U, c->ucap, c->uni, (u32)c->K_down, c->sel, ap, c->ctrl, c->ghist);
         if (rc != TK_OK) return rc;
         c->launches += 1;
     }

@@ -12,9 +12,10 @@
 //                    histograms (11+11+9 key bits, then 11+11+10 index bits, as
 //                    far as needed) and is filtered again.  Exits at once when
 //                    every row verified.
-//   select_kernel    one thread-block cluster per row: range-adaptive radix
-//                    select of the K largest composite keys among the
-//                    candidates, then emission of exactly K entries
+//   select_kernel    one thread-block cluster per row (or, for one long list, the
+//                    whole grid): range-adaptive radix select of the K largest
+//                    composite keys among the candidates, then emission of
+//                    exactly K entries
 //
 // The result is always the exact Top_K; the sample only decides how many
 // passes over the data it takes.
@@ -589,17 +590,27 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
 
 // lists[row] holds the row's candidates: exactly the entries with ck >= rs[row].lo, all with
 // key <= rs[row].max_key, rs[row].cand_count of them.
+//
+// Two ways to spread one row over several CTAs:
+//   kGrid == false  one thread-block cluster per row; the CTAs' histograms are combined
+//                   through distributed shared memory, cluster barriers between levels
+//   kGrid == true   a single row spread over the whole (cooperatively launched) grid, for
+//                   lists too long for one cluster (the union of N uplink messages);
+//                   histograms are combined in `ghist` (3 x kHistBins words of global
+//                   memory, all zero when the kernel starts), grid barriers between levels
+template <bool kGrid>
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
-              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
+              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl, u32* ghist) {
     __shared__ u32 sh_hist[2][kHistBins];  // double-buffered: peers may still read level L while L+1 fills
     __shared__ u32 sh_tot[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
     cg::cluster_group cluster = cg::this_cluster();
-    const u32 CS = cluster.num_blocks();
-    const u32 rank = cluster.block_rank();
-    const u32 row = blockIdx.x / CS;
+    cg::grid_group grid = cg::this_grid();
+    const u32 CS = kGrid ? gridDim.x : cluster.num_blocks();
+    const u32 rank = kGrid ? blockIdx.x : cluster.block_rank();
+    const u32 row = kGrid ? 0u : blockIdx.x / CS;
     RowState* r = rs + row;
     const u32 C = min(r->cand_count, cap);
     const u32 Keff = min(K, C);
@@ -648,11 +659,26 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                 u64 off = composite(key_of(e.y), e.x) - lo;
                 if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
-            cluster.sync();  // all CTAs of the row have filled this level's histogram
-            for (int b = threadIdx.x; b < nb; b += kSelectThreads) {
-                u32 sum = 0;
-                for (u32 c = 0; c < CS; ++c) sum += cluster.map_shared_rank(hist, c)[b];
-                sh_tot[b] = sum;
+            if (kGrid) {
+                u32* gh = ghist + (u32)(level % 3) * kHistBins;
+                __syncthreads();
+                for (int b = threadIdx.x; b < nb; b += kSelectThreads)
+                    if (hist[b]) atomicAdd(&gh[b], hist[b]);
+                grid.sync();  // every CTA has added its counts
+                for (int b = threadIdx.x; b < nb; b += kSelectThreads) sh_tot[b] = __ldcg(&gh[b]);
+                // the buffer read at the previous level is idle now and is not written before the
+                // next barrier: clear it for the level after next
+                if (rank == 0) {
+                    u32* idle = ghist + (u32)((level + 2) % 3) * kHistBins;
+                    for (int b = threadIdx.x; b < kHistBins; b += kSelectThreads) idle[b] = 0;
+                }
+            } else {
+                cluster.sync();  // all CTAs of the row have filled this level's histogram
+                for (int b = threadIdx.x; b < nb; b += kSelectThreads) {
+                    u32 sum = 0;
+                    for (u32 c = 0; c < CS; ++c) sum += cluster.map_shared_rank(hist, c)[b];
+                    sh_tot[b] = sum;
+                }
             }
             __syncthreads();
             u32 b, above;
@@ -674,7 +700,14 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             T = lo;
             if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
         }
-        cluster.sync();  // no CTA leaves while a peer may still read its histograms
+        if (kGrid) {
+            // leave ghist all zero for the next launch: once everybody has read the last level
+            grid.sync();
+            if (rank == 0)
+                for (int b = threadIdx.x; b < 3 * kHistBins; b += kSelectThreads) ghist[b] = 0;
+        } else {
+            cluster.sync();  // no CTA leaves while a peer may still read its histograms
+        }
     }
 
     // emission: every entry with ck >= T, exactly Keff of them; one counter update per warp
