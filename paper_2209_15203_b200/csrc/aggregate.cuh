@@ -47,11 +47,25 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         head[j] = 0;
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
     }
+    // append (j, g_j) to the union list: one counter update and one maximum per CTA (every entry
+    // of every worker passes through here; per-warp atomics on the two words would serialise)
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_base, sh_max;
+    if (threadIdx.x == 0) sh_max = 0;
     u32 bits = __float_as_uint(acc);
-    u32 m = warp_append(owner, j, bits, &uni->cand_count, U, ucap);
-    if (m) {  // the downlink selection wants the largest aggregated magnitude
-        u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
-        if ((int)lane_id() == __ffs(m) - 1) atomicMax(&uni->max_key, wm);
+    u32 owners;
+    u32 incl = block_inclusive_scan(owner ? 1u : 0u, sh_scratch, &owners);
+    u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
+    if (lane_id() == 0 && wm) atomicMax(&sh_max, wm);
+    __syncthreads();
+    if (threadIdx.x == 0 && owners) {
+        sh_base = atomicAdd(&uni->cand_count, owners);
+        atomicMax(&uni->max_key, sh_max);  // the downlink selection wants the largest aggregated magnitude
+    }
+    __syncthreads();
+    if (owner) {
+        u32 slot = sh_base + incl - 1;
+        if (slot < ucap) U[slot] = make_uint2(j, bits);
     }
 }
 

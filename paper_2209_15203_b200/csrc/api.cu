@@ -224,11 +224,19 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
     return L;
 }
 
-int cluster_size_for(int64_t entries) {
-    int64_t want = (entries + 8191) / 8192;
-    int cs = 1;
-    while (cs < 8 && cs < want) cs *= 2;
-    return cs;
+// CTAs per row of the cluster select: enough that a row's expected candidates sit in registers
+// (kSelectRegs per thread), at least 4 when there are few rows (latency), but never so many
+// that the clusters of all rows stop fitting in one wave.
+int cluster_size_for(int64_t entries, int64_t rows, int sms) {
+    int64_t per_cta = (int64_t)kSelectThreads * kSelectRegs;
+    int64_t need = (entries + per_cta - 1) / per_cta;
+    int cs_need = 1;
+    while (cs_need < 8 && cs_need < need) cs_need *= 2;
+    int cs_fill = 1;
+    while (cs_fill < 8 && (int64_t)cs_fill * 2 * rows <= sms) cs_fill *= 2;
+    int floor4 = cs_fill < 4 ? cs_fill : 4;
+    int cs = cs_need > floor4 ? cs_need : floor4;
+    return cs < cs_fill ? cs : cs_fill;
 }
 
 #define TK_LAUNCH_CHECK()                                   \
@@ -345,10 +353,10 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             *launches += 1;
         }
         ApplyArgs none = {nullptr, 0.0f};
-        int64_t expect = predict ? 3 * K : (int64_t)b.cap;
+        int64_t expect = predict ? 2 * K : (int64_t)b.cap;
         LinkArgs lk = link;
         lk.row_base = (u32)r0;
-        rc = launch_select(stream, nr, cluster_size_for(expect), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, none,
+        rc = launch_select(stream, nr, cluster_size_for(expect, nr, di->sms), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, none,
                            lk, ctrl);
         if (rc != TK_OK) return rc;
         *launches += 1;
