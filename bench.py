@@ -32,9 +32,10 @@ METRIC = "gradient elements/sec per bidirectional top_K step"
 UNIT = "elements/s"
 NOMINAL_HBM_BPS = 8e12
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch on this workload,
-# from the ncu capture summarised under profiles/ (None until captured / after the kernel changed)
-FILTER_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch, from the ncu capture
+# summarised in profiles/filter_kernel_config5_rows2.md: (992.085 + 3.72) MB for 2 of the 8 workers,
+# scaled by the rows of the launch (None for any other workload, or once the kernel has changed)
+FILTER_TRAFFIC_PER_ROW_CONFIG5 = (992.085e6 + 3.72e6) / 2
 
 
 def measured_hbm_gbs():
@@ -234,7 +235,8 @@ def main():
         k_ms = st.select_ms_sum / st.select_samples
         achieved = 4.0 * elems / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": "filter_kernel" if st.rows_general == 0 else "general_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": FILTER_TRAFFIC_BYTES,
+                "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": FILTER_TRAFFIC_PER_ROW_CONFIG5 * wl.N if (wl.cid == 5 and not args.d) else None,
                 "algorithmic_bytes": 4 * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
 
     # end to end through tk_step_host: pinned host buffers, copies inside the timed region
