@@ -32,7 +32,7 @@ def k_from_ratio(d: int, num: int, den: int) -> int:
 
 @dataclass(frozen=True)
 class Workload:
-    cid: int                      # configuration number (1..5)
+    cid: int                      # configuration number (1..5 benchmark workloads, 6..9 paper shapes)
     name: str
     N: int                        # workers (rows)
     d: int                        # vector length
@@ -72,6 +72,24 @@ def _cfg(cid: int, d: Optional[int] = None) -> Workload:
         d = d or 124_000_000
         K = k_from_ratio(d, 1, 10000)
         return Workload(5, "gpt2-small-sized", 8, d, K, (K,), 10, (1,), "gauss", 150, 1e-6, 1e-3, "uniform")
+    # Shapes of the paper's own experiments (Section 4): N in {20, 50, 100} workers, the models'
+    # parameter counts, K = d - floor((1 - 0.001) d), same K up and down.  Synthetic values.
+    if cid == 6:   # MLP [784,256,128,64,10] on Fashion-MNIST, 100 workers
+        d = d or 242_762
+        K = k_from_ratio(d, 1, 1000)
+        return Workload(6, "paper-fmnist-mlp", 100, d, K, (K,), 10, (0, 1), "student", 8, 1e-4, 1e-2, "uniform")
+    if cid == 7:   # VGG19 on CIFAR10, 20 workers
+        d = d or 20_040_522
+        K = k_from_ratio(d, 1, 1000)
+        return Workload(7, "paper-vgg19", 20, d, K, (K,), 10, (0, 1), "gauss", 40, 1e-5, 1e-2, "uniform")
+    if cid == 8:   # CNN on MNIST, 50 workers
+        d = d or 1_199_882
+        K = k_from_ratio(d, 1, 1000)
+        return Workload(8, "paper-mnist-cnn", 50, d, K, (K,), 10, (0, 1), "gauss", 8, 1e-4, 1e-2, "dirichlet")
+    if cid == 9:   # CNN on Fashion-MNIST, 20 workers: the smallest model
+        d = d or 29_034
+        K = k_from_ratio(d, 1, 1000)
+        return Workload(9, "paper-fmnist-cnn", 20, d, K, (K,), 10, (0, 1), "student", 6, 1e-4, 1e-2, "uniform")
     raise ValueError("unknown configuration %r" % cid)
 
 

@@ -90,6 +90,19 @@ def test_scaled_configs_every_step(cid, d):
     run_workload(wl, 3)
 
 
+@pytest.mark.parametrize("cid", [6, 8, 9])
+def test_paper_shaped_workloads(cid):
+    # N = 20..100 workers, d not a multiple of 4 (rows start at every alignment), tiny K
+    wl = W.workload(cid)
+    assert wl.d % 4 != 0
+    run_workload(wl, 2)
+
+
+def test_paper_vgg19_shape_one_step():
+    wl = W.workload(7)
+    run_workload(wl, 1, modes=(1,))
+
+
 def test_scaled_configs_forced_general_path():
     run_workload(W.workload(2, d=600_001, N=4), 2, force_general=True)
     run_workload(W.workload(4, d=500_000, N=6), 2, force_general=True)

@@ -16,6 +16,11 @@ def test_k_values_of_the_five_configurations():
         [30, 51, 243, 1_200, 20_041]
 
 
+def test_paper_shapes():
+    assert [(W.workload(c).N, W.workload(c).d, W.workload(c).K_up) for c in (6, 7, 8, 9)] == \
+        [(100, 242_762, 243), (20, 20_040_522, 20_041), (50, 1_199_882, 1_200), (20, 29_034, 30)]
+
+
 def test_block_layout_covers_d():
     for cid, d in ((2, 117_001), (3, 25_603), (5, 1_240_000)):
         wl = W.workload(cid, d=d)
