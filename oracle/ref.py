@@ -48,6 +48,9 @@ def _load():
         lib.ref_step.argtypes = [f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
                                  i32p, f32p, f32p, u8p, i32p, f32p, ctypes.c_void_p, ctypes.c_int]
         lib.ref_step.restype = ctypes.c_int
+        lib.ref_step_ef.argtypes = [f32p, f32p, f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
+                                    i32p, f32p, i32p, f32p, ctypes.c_void_p, ctypes.c_int]
+        lib.ref_step_ef.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -142,3 +145,45 @@ def ref_step(w, G, K_up: int, K_down: int, p, alpha: float, mode: int,
         raise ValueError("ref_step rejected its arguments")
     n = count.value
     return StepResult(w, up_idx, up_val, A, touched, msg_idx[:n].copy(), msg_val[:n].copy())
+
+
+@dataclass
+class EfResult:
+    w: np.ndarray          # updated parameters
+    eps: np.ndarray        # updated worker memories [N][d]
+    delta: Optional[np.ndarray]  # updated server memory [d] (bidirectional)
+    up_idx: np.ndarray
+    up_val: np.ndarray
+    msg_idx: np.ndarray
+    msg_val: np.ndarray
+
+
+def ref_step_ef(w, eps, delta, G, K_up: int, K_down: int, p, alpha: float, mode: int,
+                nthreads: Optional[int] = None) -> EfResult:
+    """One iteration of Algorithm 1 (mode 0) / Algorithm 2 (mode 1) with the error memories.
+    Inputs are not modified; the new w, eps, delta are returned."""
+    w = _f32(w).copy()
+    eps = _f32(eps).copy()
+    G = _f32(G)
+    p = _f32(p)
+    N, d = G.shape
+    assert w.shape == (d,) and eps.shape == (N, d) and p.shape == (N,)
+    if mode == 1:
+        delta = _f32(delta).copy()
+        assert delta.shape == (d,)
+    else:
+        delta = None
+    up_idx = np.empty((N, K_up), dtype=np.int32)
+    up_val = np.empty((N, K_up), dtype=np.float32)
+    cap = min(d, K_down if mode == 1 else N * K_up)
+    msg_idx = np.empty(cap, dtype=np.int32)
+    msg_val = np.empty(cap, dtype=np.float32)
+    count = ctypes.c_int64(0)
+    nt = default_threads() if nthreads is None else nthreads
+    rc = _load().ref_step_ef(_ptr(w), _ptr(eps), _ptr(delta), _ptr(G), N, d, K_up, K_down, _ptr(p),
+                             ctypes.c_float(alpha), mode, _ptr(up_idx), _ptr(up_val),
+                             _ptr(msg_idx), _ptr(msg_val), ctypes.byref(count), nt)
+    if rc != 0:
+        raise ValueError("ref_step_ef rejected its arguments")
+    n = count.value
+    return EfResult(w, eps, delta, up_idx, up_val, msg_idx[:n].copy(), msg_val[:n].copy())

@@ -31,6 +31,9 @@
  *               the gradient, which selects the same components because
  *               Top_K is positively homogeneous).
  *
+ *   ref_step_ef, at the end of this file, is the iteration exactly as printed,
+ *   with the error memories epsilon and delta and the step size inside a^q.
+ *
  * Magnitudes are compared through the integer key  bits(x) & 0x7fffffff,
  * which orders finite floats exactly like |x| does, makes -0 equal +0 and keeps
  * denormals distinct.  NaN/Inf are ordered by that bit pattern.
@@ -251,5 +254,87 @@ int ref_step(float *w, const float *G, int64_t N, int64_t d, int64_t K_up, int64
     rc = 0;
 done:
     free(up_idx); free(up_val); free(A); free(touched); free(msg_idx); free(msg_val);
+    return rc;
+}
+
+/*
+ * One iteration of Algorithm 1 (mode 0) or Algorithm 2 (mode 1) as printed,
+ * with the error memories: epsilon^q per worker, delta on the server.
+ *
+ *   worker q:  a^q   = epsilon^q + alpha * g^q             (first worker line)
+ *              msg^q = Top_K_up(a^q)
+ *              epsilon^q <- a^q - msg^q                     (second worker line)
+ *   server:    S = sum_q p_q msg^q   in worker order, from +0
+ *     mode 0:  g = S;            the downlink carries g;          w <- w - g
+ *     mode 1:  g = S + delta;    the downlink carries Top_K_down(g);
+ *              delta <- g - Top_K_down(g);                        w <- w - Top_K_down(g)
+ *
+ * Every operation is one rounded fp32 operation: a = fl(eps + fl(alpha*g)),
+ * S as in ref_aggregate, g = fl(S + delta), w = fl(w - msg).  Subtracting the
+ * message from a (or g) leaves exactly +0 at the sent positions and the value
+ * itself elsewhere.
+ *
+ *   w [d], eps [N][d], delta [d] (mode 1 only; may be NULL in mode 0): updated in place
+ *   G [N][d]
+ * Optional outputs as in ref_step: up_idx/up_val [N][K_up]; msg_idx/msg_val/msg_count the
+ * downlink message (mode 1: exactly K_down entries; mode 0: the union, ascending).
+ */
+int ref_step_ef(float *w, float *eps, float *delta, const float *G, int64_t N, int64_t d,
+                int64_t K_up, int64_t K_down, const float *p, float alpha, int mode,
+                int32_t *up_idx_out, float *up_val_out,
+                int32_t *msg_idx_out, float *msg_val_out, int64_t *msg_count_out, int nthreads)
+{
+    if (!w || !eps || !G || !p || N < 1 || d < 1 || K_up < 1 || K_up > d || (mode != 0 && mode != 1))
+        return -1;
+    if (mode == 1 && (!delta || K_down < 1 || K_down > d)) return -1;
+    int rc = -1;
+    int64_t cap = mode == 1 ? K_down : N * K_up;
+    if (cap > d) cap = d;
+    int32_t *up_idx = (int32_t *)malloc((size_t)(N * K_up) * sizeof *up_idx);
+    float *up_val = (float *)malloc((size_t)(N * K_up) * sizeof *up_val);
+    float *S = (float *)malloc((size_t)d * sizeof *S);
+    uint8_t *touched = (uint8_t *)malloc((size_t)d);
+    int32_t *msg_idx = (int32_t *)malloc((size_t)cap * sizeof *msg_idx);
+    float *msg_val = (float *)malloc((size_t)cap * sizeof *msg_val);
+    int64_t count = 0;
+    if (!up_idx || !up_val || !S || !touched || !msg_idx || !msg_val) goto done;
+
+    /* workers: error-compensated value, kept in eps */
+    for (int64_t q = 0; q < N; ++q)
+        for (int64_t j = 0; j < d; ++j) {
+            volatile float scaled = alpha * G[q * d + j];
+            volatile float a = eps[q * d + j] + scaled;
+            eps[q * d + j] = a;
+        }
+    if (ref_topk_rows(eps, N, d, K_up, up_idx, up_val, nthreads) != 0) goto done;
+    /* eps <- a - Top_K(a) */
+    for (int64_t q = 0; q < N; ++q)
+        for (int64_t k = 0; k < K_up; ++k) eps[q * d + up_idx[q * K_up + k]] = 0.0f;
+    /* server */
+    if (ref_aggregate(up_idx, up_val, N, K_up, p, d, S, touched) != 0) goto done;
+    if (mode == 1) {
+        for (int64_t j = 0; j < d; ++j) {
+            volatile float g = S[j] + delta[j];
+            delta[j] = g;
+        }
+        if (ref_topk(delta, d, K_down, msg_idx, msg_val) != 0) goto done;
+        count = K_down;
+        for (int64_t k = 0; k < count; ++k) delta[msg_idx[k]] = 0.0f;
+    } else {
+        for (int64_t j = 0; j < d; ++j)
+            if (touched[j]) { msg_idx[count] = (int32_t)j; msg_val[count] = S[j]; ++count; }
+    }
+    for (int64_t k = 0; k < count; ++k) {
+        volatile float nw = w[msg_idx[k]] - msg_val[k];
+        w[msg_idx[k]] = nw;
+    }
+    if (up_idx_out) memcpy(up_idx_out, up_idx, (size_t)(N * K_up) * sizeof *up_idx);
+    if (up_val_out) memcpy(up_val_out, up_val, (size_t)(N * K_up) * sizeof *up_val);
+    if (msg_idx_out) memcpy(msg_idx_out, msg_idx, (size_t)count * sizeof *msg_idx);
+    if (msg_val_out) memcpy(msg_val_out, msg_val, (size_t)count * sizeof *msg_val);
+    if (msg_count_out) *msg_count_out = count;
+    rc = 0;
+done:
+    free(up_idx); free(up_val); free(S); free(touched); free(msg_idx); free(msg_val);
     return rc;
 }
