@@ -59,7 +59,9 @@ enum {
 
 enum {
     TK_MODE_UNI = 0,   /* Algorithm 1: the downlink carries the aggregate itself */
-    TK_MODE_BIDIR = 1  /* Algorithm 2: the downlink carries Top_K_down of the aggregate */
+    TK_MODE_BIDIR = 1, /* Algorithm 2: the downlink carries Top_K_down of the aggregate */
+    TK_MODE_EF = 2     /* flag, OR-ed in: keep the error memories epsilon^q and delta of
+                          Algorithm 1/2 as printed (see tk_ef_attach) */
 };
 
 /* Counters of the last step / selection, filled by tk_status(). */
@@ -102,7 +104,7 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down,
  *   w_dev      [d]     parameters, updated in place
  *   grads_dev  [N][d]  the workers' vectors, read only
  *   alpha      finite step size
- *   mode       TK_MODE_UNI or TK_MODE_BIDIR
+ *   mode       TK_MODE_UNI or TK_MODE_BIDIR, optionally | TK_MODE_EF (error memories, below)
  * Asynchronous.  Inputs are assumed finite.
  */
 int tk_step(tk_ctx* ctx, float* w_dev, const float* grads_dev, float alpha, int mode);
@@ -164,6 +166,34 @@ int tk_topk(tk_ctx* ctx, const float* x_dev, int32_t rows, int64_t d, int64_t K,
 #define TK_NOALLOC_SCRATCH_BYTES (4u << 20)
 int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
                     float* val_out_dev, void* cuda_stream);
+
+/*
+ * Error memories: the iteration exactly as Algorithm 1 / Algorithm 2 print it.
+ *
+ * With TK_MODE_EF set in `mode`, tk_step(w, grads, alpha, mode) does
+ *   worker q:  a^q = epsilon^q + alpha * g^q;  SEND(Top_K_up(a^q));  epsilon^q <- a^q - Top_K_up(a^q)
+ *   server:    S = sum_q p_q Top_K_up(a^q)  (worker order, from +0)
+ *     TK_MODE_UNI | TK_MODE_EF    g = S, sent as it is;                     w <- w - g
+ *     TK_MODE_BIDIR | TK_MODE_EF  g = S + delta; SEND(Top_K_down(g));
+ *                                 delta <- g - Top_K_down(g);               w <- w - Top_K_down(g)
+ * (the step size sits inside a^q, as in the paper; one rounding per multiply / add / subtract).
+ * The memories live in device memory the caller provides once:
+ *   tk_ef_bytes   bytes needed for N worker memories [N][d], the server memory [d] and the
+ *                 scratch of the selection over the dense server vector (0 if the sizes are invalid)
+ *   tk_ef_attach  mem_dev: at least tk_ef_bytes(d, N, K_down of the context) bytes, 256-byte
+ *                 aligned, caller-owned, alive until tk_destroy; sets epsilon = delta = 0 (the
+ *                 initialisation line of the algorithms) and synchronises.  Attaching again
+ *                 restarts the memories.  After tk_set_kdown to a LARGER K_down, attach again
+ *                 before the next TK_MODE_EF step (it is refused otherwise).
+ *   tk_ef_state   device pointers to epsilon [N][d] and delta [d] (for checkpoints and tests;
+ *                 stream-ordered with the steps).  Either output may be NULL.
+ * tk_last_aggregate then reports S (without delta); tk_last_downlink the message sent.
+ * Per step this path moves 12 bytes per gradient value (read g, read and write epsilon)
+ * instead of 4, plus one pass over the d-long server vector when bidirectional.
+ */
+size_t tk_ef_bytes(int64_t d, int32_t N, int64_t K_down);
+int tk_ef_attach(tk_ctx* ctx, void* mem_dev, size_t bytes);
+int tk_ef_state(tk_ctx* ctx, float** eps_dev, float** delta_dev);
 
 /* Change K_downlink of an existing context (1 <= K_down <= d). */
 int tk_set_kdown(tk_ctx* ctx, int64_t K_down);

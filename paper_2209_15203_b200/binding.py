@@ -18,8 +18,10 @@ from . import build as _build
 
 TK_MODE_UNI = 0
 TK_MODE_BIDIR = 1
+TK_MODE_EF = 2
 
-EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_set_kdown",
+EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
+           "tk_ef_attach", "tk_ef_state", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
            "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
@@ -67,6 +69,12 @@ def load(build_if_missing: bool = True):
     lib.tk_topk.argtypes = [vp, vp, i32, i64, i64, vp, vp]
     lib.tk_topk_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, vp]
     lib.tk_topk_noalloc.restype = ctypes.c_int
+    lib.tk_ef_bytes.argtypes = [i64, i32, i64]
+    lib.tk_ef_bytes.restype = ctypes.c_size_t
+    lib.tk_ef_attach.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.tk_ef_attach.restype = ctypes.c_int
+    lib.tk_ef_state.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.tk_ef_state.restype = ctypes.c_int
     lib.tk_set_kdown.argtypes = [vp, i64]
     lib.tk_last_uplink.argtypes = [vp, vp, vp]
     lib.tk_last_aggregate.argtypes = [vp, vp, vp, ctypes.POINTER(i64)]
@@ -160,6 +168,25 @@ class Context:
     def tk_topk(self, x: torch.Tensor, K: int) -> Tuple[torch.Tensor, torch.Tensor]:
         return tk_topk(x, K, ctx=self)
 
+    def tk_ef_attach(self) -> None:
+        """Allocate (with torch) and attach the error memories; epsilon = delta = 0."""
+        lib = load()
+        nbytes = int(lib.tk_ef_bytes(self.d, self.N, self.K_down))
+        if nbytes == 0:
+            raise TkError(-1, "tk_ef_bytes")
+        with torch.cuda.device(self.device):
+            self.ef_memory = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            _check(lib.tk_ef_attach(self._h, self.ef_memory.data_ptr(), nbytes), "tk_ef_attach")
+
+    def tk_ef_state(self) -> Tuple[torch.Tensor, torch.Tensor]:
+        """Views of epsilon [N][d] and delta [d] inside the attached memory."""
+        e, dl = ctypes.c_void_p(), ctypes.c_void_p()
+        _check(load().tk_ef_state(self._h, ctypes.byref(e), ctypes.byref(dl)), "tk_ef_state")
+        base = self.ef_memory.data_ptr()
+        flat = self.ef_memory.view(torch.float32)
+        eo, do = (e.value - base) // 4, (dl.value - base) // 4
+        return flat[eo:eo + self.N * self.d].view(self.N, self.d), flat[do:do + self.d]
+
     def tk_set_kdown(self, K_down: int) -> None:
         _check(load().tk_set_kdown(self._h, K_down), "tk_set_kdown")
         self.K_down = K_down
@@ -181,7 +208,7 @@ class Context:
         return self._msg(load().tk_last_aggregate, "tk_last_aggregate", self.ucap)
 
     def tk_last_downlink(self) -> Tuple[torch.Tensor, torch.Tensor]:
-        n = self.K_down if self.last_mode == TK_MODE_BIDIR else self.ucap
+        n = self.K_down if (self.last_mode is not None and self.last_mode & TK_MODE_BIDIR) else self.ucap
         return self._msg(load().tk_last_downlink, "tk_last_downlink", max(n, 1))
 
     def tk_status(self, check: bool = True) -> tk_stats:

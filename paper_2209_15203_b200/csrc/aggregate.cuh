@@ -10,6 +10,7 @@
 // append (j, g_j) to the union list U, put the word back to zero, and — in
 // unidirectional mode, where the downlink carries g itself — apply
 // w_j <- w_j - alpha g_j  right there (last worker step of Algorithm 1).
+// With the server memory of Algorithm 2 it adds the sum into delta instead.
 // The work is O(N K_up); no pass over the d coordinates is ever made.
 #pragma once
 
@@ -20,7 +21,7 @@ namespace tk {
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
                   u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
-                  uint2* U, u32 ucap, float* w, float alpha, int apply, Ctrl* ctrl, u32 d) {
+                  uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d) {
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
     u32 j = 0;
@@ -46,6 +47,9 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         }
         head[j] = 0;
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
+        // server memory (Algorithm 2): g = sum + delta, kept in the memory until the downlink
+        // selection takes its Top_K out of it
+        if (delta) delta[j] = __fadd_rn(acc, delta[j]);
     }
     // append (j, g_j) to the union list: one counter update and one maximum per CTA (every entry
     // of every worker passes through here; per-warp atomics on the two words would serialise)

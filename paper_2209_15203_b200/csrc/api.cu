@@ -60,12 +60,13 @@ struct SelectBufs {
     uint2* out = nullptr;     // [rows][K]
     u32 cap = 0;
     u32 tpr_filter = 0;       // tiles per row of the filter kernel / of the multi-pass kernel
+    u32 tpr_filter_ef = 0;    // ... of the filter kernel with error memories (smaller tiles)
     u32 tpr_general = 0;
 };
 
 struct SelectLayout {
     size_t off_rs, off_hist, off_smax, off_cand, off_out, bytes;
-    u32 cap, tpr_filter, tpr_general;
+    u32 cap, tpr_filter, tpr_filter_ef, tpr_general;
 };
 
 u32 candidate_capacity(int64_t d, int64_t K) {
@@ -79,7 +80,9 @@ SelectLayout select_layout(int64_t rows, int64_t d, int64_t K) {
     L.cap = candidate_capacity(d, K);
     int64_t nv = (d + 3) / 4;
     int64_t tf = (nv + kFilterTileVecs - 1) / kFilterTileVecs, tg = (nv + kGeneralTileVecs - 1) / kGeneralTileVecs;
+    int64_t te = (nv + kFilterEfTileVecs - 1) / kFilterEfTileVecs;
     L.tpr_filter = (u32)(tf < 1 ? 1 : tf);
+    L.tpr_filter_ef = (u32)(te < 1 ? 1 : te);
     L.tpr_general = (u32)(tg < 1 ? 1 : tg);
     size_t o = 0;
     L.off_rs = o;   o += align_up((size_t)rows * sizeof(RowState));
@@ -100,6 +103,7 @@ SelectBufs bind(const SelectLayout& L, char* base) {
     b.out = (uint2*)(base + L.off_out);
     b.cap = L.cap;
     b.tpr_filter = L.tpr_filter;
+    b.tpr_filter_ef = L.tpr_filter_ef;
     b.tpr_general = L.tpr_general;
     return b;
 }
@@ -190,6 +194,11 @@ struct tk_ctx {
     int ev_used = 0;
     float* stage_g = nullptr;  // tk_step_host staging
     float* stage_w = nullptr;
+    // error memories (tk_ef_attach)
+    float* eps = nullptr;      // [N][d]
+    float* delta = nullptr;    // [d]
+    SelectBufs down;           // selection over the dense server vector (1 row of d)
+    int64_t ef_kdown = 0;      // largest K_down the attached buffers serve
 };
 
 namespace {
@@ -285,13 +294,29 @@ int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap
 
 // Exact Top_K of every row of x into b.out ([rows][K], arbitrary order).  ev0/ev1, when
 // given, bracket the streaming pass.  *launches is advanced by the kernels enqueued.
+//
+// With error memories (ef.eps != NULL) the vector selected from is a = eps + alpha*x, which
+// also replaces eps; the streaming pass computes it on the fly when x and eps are equally
+// aligned, otherwise a separate pass does and the selection then reads eps alone.
 int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
                Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches,
-               RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0}) {
+               RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0},
+               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}) {
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
     const bool predict = !force_general && d >= 262144 && K * 64 <= d;
+    bool fused = ef.eps != nullptr && predict && ((((uintptr_t)x) ^ ((uintptr_t)ef.eps)) & 15u) == 0;
+    if (ef.eps && !fused) {
+        size_t n = (size_t)rows * (size_t)d;
+        size_t blocks = (n + 1023) / 1024;
+        if (blocks > (size_t)di->sms * 16) blocks = (size_t)di->sms * 16;
+        compensate_kernel<<<(unsigned)blocks, 256, 0, stream>>>(ef.eps, x, ef.alpha, n);
+        TK_LAUNCH_CHECK();
+        *launches += 1;
+        x = ef.eps;            // from here on this is an ordinary selection over eps
+        ef.eps = nullptr;
+    }
     int turns = 1;
     u64 stride_fp = 0;
     u32 rank = 0;
@@ -299,8 +324,9 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         // sample ~128*d/K values per row (about 128 members of the top K; fewer when that would take
         // more than kPredictMaxTurns loads per thread), as whole 128-byte lines
         const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
+        const int64_t max_turns = fused ? kPredictMaxTurns / 2 : kPredictMaxTurns;
         int64_t want = (128 * (d / K) + per_turn - 1) / per_turn;
-        int64_t lim = d / (8 * per_turn) < kPredictMaxTurns ? d / (8 * per_turn) : kPredictMaxTurns;
+        int64_t lim = d / (8 * per_turn) < max_turns ? d / (8 * per_turn) : max_turns;
         turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
         if (turns < 1) turns = 1;
         u64 lines = (u64)turns * (2 * kSampleSlots / 8);
@@ -317,20 +343,32 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         u32* smax = b.smax + (size_t)r0 * kSampleSlots;
         uint2* cand = b.cand + (size_t)r0 * b.cap;
         uint2* out = b.out + (size_t)r0 * (size_t)K;
+        EfArgs efb = {fused ? ef.eps + (size_t)r0 * (size_t)d : nullptr, ef.alpha};
         if (predict) {
-            predict_kernel<<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs,
-                                                                                   smax, r0 == 0 ? also_reset : nullptr);
+            RowState* ar = r0 == 0 ? also_reset : nullptr;
+            if (fused)
+                predict_kernel<true><<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank,
+                                                                                             rs, smax, ar, efb);
+            else
+                predict_kernel<false><<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank,
+                                                                                              rs, smax, ar, efb);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
-            u64 tiles = (u64)nr * b.tpr_filter;
+            u32 tprf = fused ? b.tpr_filter_ef : b.tpr_filter;
+            u64 tiles = (u64)nr * tprf;
             u64 resident = (u64)di->sms * kFilterCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
             u32 grid = (u32)(tiles < resident ? tiles : resident);
             u32 parts = 1;
             if (tiles >= 4 * resident) parts = (u32)(nr < kFilterPartitions ? nr : kFilterPartitions);
             u32 cpp = grid / parts;
-            filter_kernel<<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, b.tpr_filter, parts, cpp,
-                                                                                        rs, cand, b.cap);
+            if (fused)
+                filter_kernel<true><<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, tprf, parts, cpp,
+                                                                                              rs, cand, b.cap, efb);
+            else
+                filter_kernel<false><<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, tprf, parts, cpp,
+                                                                                               rs, cand, b.cap, efb);
             TK_LAUNCH_CHECK();
+            if (fused) xb = efb.eps;  // the compensated vector now sits in eps: what a re-filter must read
             if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 2;
         } else {
@@ -352,11 +390,11 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             if (!predict && ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 1;
         }
-        ApplyArgs none = {nullptr, 0.0f};
         int64_t expect = predict ? 2 * K : (int64_t)b.cap;
         LinkArgs lk = link;
         lk.row_base = (u32)r0;
-        rc = launch_select(stream, nr, cluster_size_for(expect, nr, di->sms), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, none,
+        if (lk.zero_src) lk.zero_src += (size_t)r0 * lk.zero_stride;
+        rc = launch_select(stream, nr, cluster_size_for(expect, nr, di->sms), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, apply,
                            lk, ctrl);
         if (rc != TK_OK) return rc;
         *launches += 1;
@@ -460,7 +498,9 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
 
 int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
     if (!c || !aligned4(w_dev) || !aligned4(grads_dev) || !isfinite(alpha)) return TK_ERR_INVALID;
-    if (mode != TK_MODE_UNI && mode != TK_MODE_BIDIR) return TK_ERR_INVALID;
+    if (mode < 0 || mode > (TK_MODE_BIDIR | TK_MODE_EF)) return TK_ERR_INVALID;
+    const bool bidir = (mode & TK_MODE_BIDIR) != 0, with_ef = (mode & TK_MODE_EF) != 0;
+    if (with_ef && (!c->eps || c->K_down > c->ef_kdown)) return TK_ERR_INVALID;
     cudaStream_t s = c->stream;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
@@ -469,18 +509,31 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
         c->ev_used += 1;
     }
     // the first kernel of the selection also resets the state of the union / downlink selection
-    // ... and its last kernel threads every uplink entry onto its coordinate's chain
-    LinkArgs link = {c->head, c->next, (u32)c->d, 0};
+    // ... and its last kernel threads every uplink entry onto its coordinate's chain (and, with
+    // error memories, zeroes the sent entries in eps)
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d};
+    EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
     int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
-                        &c->launches, c->uni, link);
+                        &c->launches, c->uni, link, ef);
     if (rc != TK_OK) return rc;
+    // with memories the step size is already inside the messages
+    const float scale = with_ef ? 1.0f : alpha;
     u32 total = (u32)(c->N * c->K_up);
     u32 blocks = (total + 255) / 256;
     agg_reduce_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->uni, c->U,
-                                             c->ucap, w_dev, alpha, mode == TK_MODE_UNI ? 1 : 0, c->ctrl, (u32)c->d);
+                                             c->ucap, w_dev, scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : nullptr,
+                                             c->ctrl, (u32)c->d);
     TK_LAUNCH_CHECK();
     c->launches += 1;
-    if (mode == TK_MODE_BIDIR) {
+    if (bidir && with_ef) {
+        // Algorithm 2 with the server memory: delta now holds g = sum + delta everywhere; take
+        // Top_K_down out of it (delta <- g - Top_K(g)) and apply it (w <- w - Top_K(g))
+        LinkArgs zero = {nullptr, nullptr, 0, 0, c->delta, (size_t)c->d};
+        ApplyArgs ap = {w_dev, 1.0f};
+        rc = run_select(s, c->delta, 1, c->d, c->K_down, c->down, c->ctrl, c->force_general != 0, nullptr, nullptr,
+                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap);
+        if (rc != TK_OK) return rc;
+    } else if (bidir) {
         ApplyArgs ap = {w_dev, alpha};
         DeviceInfo* di = nullptr;
         rc = device_info(&di);
@@ -547,6 +600,43 @@ int tk_topk(tk_ctx* c, const float* x_dev, int32_t rows, int64_t d, int64_t K, i
                     (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, launches);
 }
 
+size_t tk_ef_bytes(int64_t d, int32_t N, int64_t K_down) {
+    if (!sizes_ok(d, N, 1, K_down)) return 0;
+    size_t rows = align_up((size_t)N * (size_t)d * sizeof(float));
+    return rows + align_up((size_t)d * sizeof(float)) + select_layout(1, d, K_down).bytes;
+}
+
+int tk_ef_attach(tk_ctx* c, void* mem_dev, size_t bytes) {
+    if (!c || !mem_dev || ((uintptr_t)mem_dev & (kAlign - 1)) != 0) return TK_ERR_INVALID;
+    size_t need = tk_ef_bytes(c->d, c->N, c->K_down);
+    if (need == 0 || bytes < need) return TK_ERR_ALLOC;
+    char* base = (char*)mem_dev;
+    size_t off_delta = align_up((size_t)c->N * (size_t)c->d * sizeof(float));
+    size_t off_down = off_delta + align_up((size_t)c->d * sizeof(float));
+    SelectLayout L = select_layout(1, c->d, c->K_down);
+    SelectBufs down = bind(L, base + off_down);
+    // epsilon_0 = delta_0 = 0 (initialisation line of Algorithm 1/2); selection state zero at rest
+    if (cudaMemsetAsync(base, 0, off_down, c->stream) != cudaSuccess ||
+        cudaMemsetAsync(down.rs, 0, sizeof(RowState), c->stream) != cudaSuccess ||
+        cudaMemsetAsync(down.hist, 0, (size_t)kHistBins * sizeof(u32), c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    c->eps = (float*)base;
+    c->delta = (float*)(base + off_delta);
+    c->down = down;
+    c->ef_kdown = c->K_down;
+    return TK_OK;
+}
+
+int tk_ef_state(tk_ctx* c, float** eps_dev, float** delta_dev) {
+    if (!c || !c->eps) return TK_ERR_INVALID;
+    if (eps_dev) *eps_dev = c->eps;
+    if (delta_dev) *delta_dev = c->delta;
+    return TK_OK;
+}
+
 int tk_set_kdown(tk_ctx* c, int64_t K_down) {
     if (!c || K_down < 1 || K_down > c->d) return TK_ERR_INVALID;
     c->K_down = K_down;
@@ -588,8 +678,21 @@ int tk_last_aggregate(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64
 
 int tk_last_downlink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64_t* count_host) {
     if (!c || c->last_mode < 0) return TK_ERR_INVALID;
-    if (c->last_mode == TK_MODE_UNI) return tk_last_aggregate(c, idx_out_dev, val_out_dev, count_host);
+    if (!(c->last_mode & TK_MODE_BIDIR)) return tk_last_aggregate(c, idx_out_dev, val_out_dev, count_host);
     if (!aligned4(idx_out_dev) || !aligned4(val_out_dev) || !count_host) return TK_ERR_INVALID;
+    if (c->last_mode & TK_MODE_EF) {
+        // selected from the dense server vector: already the exact K_down-entry message
+        u32 Kd = (u32)c->last_kdown;
+        SortLayout QL = sort_layout(1, Kd);
+        char* base = nullptr;
+        int rc = pool_get(QL.bytes, &base);
+        if (rc != TK_OK) return rc;
+        *count_host = Kd;
+        rc = run_sort(c->stream, c->down.out, Kd, nullptr, 0, Kd, 1, c->d, (uint2*)(base + QL.off_tmp),
+                      (u32*)(base + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, Kd, &c->launches);
+        if (rc != TK_OK) return rc;
+        return cudaStreamSynchronize(c->stream) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+    }
     // The step selects among the union only.  The message proper has exactly K_down entries:
     // every selected entry of non-zero magnitude, then zero-valued entries at the lowest
     // indices that carry no such entry.
@@ -656,7 +759,8 @@ int tk_status(tk_ctx* c, tk_stats* out) {
     out->device_status = ctrl.status;
     out->rows_general = (int32_t)ctrl.rows_general;
     out->union_size = u.cand_count;
-    out->downlink_count = c->last_mode == TK_MODE_BIDIR ? u.out_count : u.cand_count;
+    out->downlink_count = (c->last_mode >= 0 && (c->last_mode & TK_MODE_BIDIR)) ? u.out_count : u.cand_count;
+    if (c->last_mode == (TK_MODE_BIDIR | TK_MODE_EF)) out->downlink_count = c->last_kdown;
     int64_t lo = INT64_MAX, hi = 0;
     for (int q = 0; q < c->N; ++q) {
         int64_t v = rows[q].cand_count;

@@ -45,6 +45,8 @@ constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads
 constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
 constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
+constexpr int kFilterEfUnroll = 3;     // with error memories a thread has two loads in flight per float4
+constexpr int kFilterEfTileVecs = kFilterThreads * kFilterEfUnroll;
 constexpr int kFilterPartitions = 8;   // the filter grid splits the tile space into this many ranges
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 constexpr int kMaxRowsPerLaunch = 4096;
@@ -79,6 +81,26 @@ __device__ __forceinline__ u64 composite(u32 key, u32 idx) {
 
 __device__ __forceinline__ void raise_status(Ctrl* ctrl, int code) {
     atomicCAS(&ctrl->status, 0, code);
+}
+
+// The vector a worker compresses.  Memory-free iteration: its gradient g.  With error
+// memories (first worker line of Algorithm 1/2): a = eps + alpha * g, one rounding each.
+struct EfArgs {
+    float* eps;   // [rows][d] worker memories, NULL for the memory-free iteration
+    float alpha;
+};
+
+__device__ __forceinline__ u32 compensated(u32 g_bits, u32 eps_bits, float alpha) {
+    return __float_as_uint(__fadd_rn(__uint_as_float(eps_bits), __fmul_rn(alpha, __uint_as_float(g_bits))));
+}
+
+// 16-byte streaming load of data this kernel also writes (no L1 allocation, coherent path).
+__device__ __forceinline__ uint4 ld_once(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
 }
 
 // 16-byte read-only streaming load that does not allocate in L1.

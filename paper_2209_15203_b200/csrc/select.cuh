@@ -48,9 +48,10 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->g_active = 0;
 }
 
+template <bool kEF>
 __global__ void __launch_bounds__(kPredictThreads)
 predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank,
-               RowState* rs, u32* smax, RowState* also_reset) {
+               RowState* rs, u32* smax, RowState* also_reset, EfArgs ef) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
@@ -59,26 +60,43 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;   // 0 .. 2*kSampleSlots-1
     if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
     const float* xr = x + (size_t)row * (size_t)d;
-    const bool vec_ok = (((uintptr_t)xr) & 15u) == 0;  // runs start at multiples of 32 elements
+    const float* er = kEF ? ef.eps + (size_t)row * (size_t)d : nullptr;
+    // runs start at multiples of 32 elements
+    const bool vec_ok = (((uintptr_t)xr) & 15u) == 0 && (!kEF || (((uintptr_t)er) & 15u) == 0);
     constexpr u32 kLinesPerTurn = 2 * kSampleSlots / 8;
-    uint4 v[kPredictMaxTurns];
+    constexpr int kTurns = kEF ? kPredictMaxTurns / 2 : kPredictMaxTurns;  // two loads per turn with memories
+    uint4 v[kTurns], m[kEF ? kTurns : 1];
 #pragma unroll
-    for (int k = 0; k < kPredictMaxTurns; ++k) {
+    for (int k = 0; k < kTurns; ++k) {
         v[k] = make_uint4(0, 0, 0, 0);
+        if (kEF) m[k] = make_uint4(0, 0, 0, 0);
         if (k < turns) {
             u64 g = (u64)(t >> 3) + (u64)k * kLinesPerTurn;
             u64 e = (((g * stride_fp) >> 32) & ~31ull) + 4u * (t & 7u);
             if (vec_ok) {
                 v[k] = ld_stream(reinterpret_cast<const uint4*>(xr + e));
+                if (kEF) m[k] = ld_stream(reinterpret_cast<const uint4*>(er + e));
             } else {
                 v[k] = make_uint4(__float_as_uint(__ldg(xr + e)), __float_as_uint(__ldg(xr + e + 1)),
                                   __float_as_uint(__ldg(xr + e + 2)), __float_as_uint(__ldg(xr + e + 3)));
+                if (kEF)
+                    m[k] = make_uint4(__float_as_uint(__ldg(er + e)), __float_as_uint(__ldg(er + e + 1)),
+                                      __float_as_uint(__ldg(er + e + 2)), __float_as_uint(__ldg(er + e + 3)));
             }
+        }
+    }
+    if (kEF) {
+#pragma unroll
+        for (int k = 0; k < kTurns; ++k) {
+            v[k].x = compensated(v[k].x, m[k].x, ef.alpha);
+            v[k].y = compensated(v[k].y, m[k].y, ef.alpha);
+            v[k].z = compensated(v[k].z, m[k].z, ef.alpha);
+            v[k].w = compensated(v[k].w, m[k].w, ef.alpha);
         }
     }
     u32 mx = 0;
 #pragma unroll
-    for (int k = 0; k < kPredictMaxTurns; ++k)
+    for (int k = 0; k < kTurns; ++k)
         mx = max(mx, max(max(key_of(v[k].x), key_of(v[k].y)), max(key_of(v[k].z), key_of(v[k].w))));
     mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     if ((t & 1u) == 0) smax[(size_t)row * kSampleSlots + (t >> 1)] = mx;
@@ -118,6 +136,13 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
         need -= above;
     }
     if (threadIdx.x == 0) reset_state(rs + row, (u64)prefix << 32, 0u);
+}
+
+// eps <- eps + alpha * g over n values (the compensated vector, for the paths that do not
+// fuse it into the filter pass).
+__global__ void __launch_bounds__(256) compensate_kernel(float* eps, const float* __restrict__ g, float alpha, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        eps[i] = __fadd_rn(eps[i], __fmul_rn(alpha, __ldg(g + i)));
 }
 
 // No prediction: mark every row for the multi-pass path.
@@ -250,32 +275,51 @@ __device__ __forceinline__ bool may_hit(uint4 v, float thr) {
            (!(fabsf(__uint_as_float(v.z)) < thr)) | (!(fabsf(__uint_as_float(v.w)) < thr));
 }
 
-// Process tile `tile` (THREADS * kStreamUnroll float4) of a row.  All THREADS threads of the CTA call.
-template <int THREADS>
+// Process tile `tile` (THREADS * UNROLL float4) of a row.  All THREADS threads of the CTA call.
+// With kEF the row's memory `erow` is read as well, the compensated vector a = eps + alpha*g
+// is what gets filtered, and it is written back to the memory (the entries sent later are
+// zeroed there by the selection's emission: eps <- a - Top_K(a)).
+template <int THREADS, int UNROLL, bool kEF>
 __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
-                                            RowState* rs, uint2* cand, u32 cap) {
+                                            RowState* rs, uint2* cand, u32 cap, float* erow = nullptr,
+                                            float alpha = 0.0f) {
     const u32 tk = (u32)(lo >> 32);
     const float thr = __uint_as_float(tk);
-    const u32 j0 = tile * (THREADS * kStreamUnroll) + threadIdx.x;
+    const u32 j0 = tile * (THREADS * UNROLL) + threadIdx.x;
     const uint4* p = g.vec + j0;
-    uint4 v[kStreamUnroll];
-    bool inb[kStreamUnroll];
-    const bool full = (tile + 1) * (u32)(THREADS * kStreamUnroll) <= g.nv;
+    uint4* pe = kEF ? reinterpret_cast<uint4*>(erow + g.head) + j0 : nullptr;
+    uint4 v[UNROLL];
+    uint4 m[kEF ? UNROLL : 1];
+    bool inb[UNROLL];
+    const bool full = (tile + 1) * (u32)(THREADS * UNROLL) <= g.nv;
     if (full) {
 #pragma unroll
-        for (int u = 0; u < kStreamUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             v[u] = ld_stream(p + u * THREADS);
+            if (kEF) m[u] = ld_once(pe + u * THREADS);
             inb[u] = true;
         }
     } else {
 #pragma unroll
-        for (int u = 0; u < kStreamUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
             inb[u] = j0 + u * THREADS < g.nv;
             v[u] = inb[u] ? ld_stream(p + u * THREADS) : make_uint4(0, 0, 0, 0);
+            if (kEF) m[u] = inb[u] ? ld_once(pe + u * THREADS) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    if (kEF) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            v[u].x = compensated(v[u].x, m[u].x, alpha);
+            v[u].y = compensated(v[u].y, m[u].y, alpha);
+            v[u].z = compensated(v[u].z, m[u].z, alpha);
+            v[u].w = compensated(v[u].w, m[u].w, alpha);
+            if (inb[u]) __stcs(pe + u * THREADS, v[u]);
+            else v[u] = make_uint4(0, 0, 0, 0);
         }
     }
 #pragma unroll
-    for (int u = 0; u < kStreamUnroll; ++u) {
+    for (int u = 0; u < UNROLL; ++u) {
         bool hit = inb[u] && may_hit(v[u], thr);
         if (__any_sync(0xffffffffu, hit)) {
             u32 i0 = g.head + 4u * (j0 + u * THREADS);
@@ -296,6 +340,10 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
         if (lane < g.head) { live = true; idx = lane; }
         else if (lane >= 8 && lane - 8 < g.tail) { live = true; idx = g.head + 4u * g.nv + (lane - 8); }
         u32 bits = live ? __float_as_uint(__ldg(g.base + idx)) : 0u;
+        if (kEF && live) {
+            bits = compensated(bits, __float_as_uint(erow[idx]), alpha);
+            erow[idx] = __uint_as_float(bits);
+        }
         consider(live, idx, bits, lo, st, rs, cand, cap);
     }
 }
@@ -305,9 +353,11 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
 // range every CTA would visit every row, and each change of row costs a flush of the
 // staged candidates (a global atomic round trip); with one range per CTA a CTA that
 // lands in a layer full of candidates would finish late.
+template <bool kEF>
 __global__ void __launch_bounds__(kFilterThreads, kFilterCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 parts, u32 cpp,
-              RowState* rs, uint2* cand, u32 cap) {
+              RowState* rs, uint2* cand, u32 cap, EfArgs ef) {
+    constexpr int kUnroll = kEF ? kFilterEfUnroll : kStreamUnroll;
     extern __shared__ u64 sh_lo[];  // every row's bound, fetched once
     __shared__ uint2 sh_buf[(kFilterThreads / 32) * kStageSlots];
     __shared__ u32 sh_n[kFilterThreads / 32];
@@ -332,8 +382,9 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
             g = row_geom(x, row, d);
             lo = sh_lo[row];
         }
-        if (tile * (u32)kFilterTileVecs < g.nv || tile == 0)
-            filter_tile<kFilterThreads>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        if (tile * (u32)(kFilterThreads * kUnroll) < g.nv || tile == 0)
+            filter_tile<kFilterThreads, kUnroll, kEF>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap,
+                                                      kEF ? ef.eps + (size_t)row * (size_t)d : nullptr, ef.alpha);
         tile += cpp;
         while (tile >= tpr) { tile -= tpr; ++row; }
     }
@@ -548,7 +599,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
             lo = rs[row].lo;
         }
         if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile<kGeneralThreads>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        filter_tile<kGeneralThreads, kStreamUnroll, false>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
     }
     if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
 }
@@ -568,6 +619,11 @@ struct LinkArgs {
     u32* next;
     u32 d;
     u32 row_base;  // entry ids count rows from here (rows are processed in batches)
+    // Error memories: if zero_src is non-NULL the vector the entries were taken from,
+    // zero_src[row][idx] with rows zero_stride apart, is set to +0 at every emitted entry
+    // (eps <- a - Top_K(a), delta <- g - Top_K(g): second worker / server line of Algorithm 1/2).
+    float* zero_src;
+    size_t zero_stride;
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
@@ -581,6 +637,7 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
         float upd = __fmul_rn(apply.alpha, __uint_as_float(bits));
         apply.w[idx] = __fsub_rn(apply.w[idx], upd);
     }
+    if (link.zero_src) link.zero_src[(size_t)row * link.zero_stride + idx] = 0.0f;
     if (link.head) {
         u32 e = (link.row_base + row) * (u32)out_stride + slot;
         if (idx < link.d) link.next[e] = atomicExch(&link.head[idx], e + 1);
