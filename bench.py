@@ -162,6 +162,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows", type=int, default=0, help="override the number of workers N (smaller case for profiling)")
     ap.add_argument("--d", type=int, default=0, help="override the vector length d (smaller case for profiling)")
+    ap.add_argument("--ef", action="store_true", help="keep the error memories (Algorithm 2 as printed): "
+                    "12 bytes per gradient value instead of 4")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -196,7 +198,9 @@ def main():
     bufs = [W.make_grads(wl, s, dev, scale=scale) for s in range(nbuf)]
     del scale
     w = W.make_w(wl, dev)
-    mode = binding.TK_MODE_BIDIR
+    mode = binding.TK_MODE_BIDIR | (binding.TK_MODE_EF if args.ef else 0)
+    if args.ef:
+        ctx.tk_ef_attach()
 
     def barrier():
         replicas.barrier()
@@ -233,11 +237,12 @@ def main():
     roof = None
     if st.select_samples > 0 and st.select_ms_sum > 0:
         k_ms = st.select_ms_sum / st.select_samples
-        achieved = 4.0 * elems / (k_ms * 1e-3) / 1e9
+        bytes_per_elem = 12.0 if args.ef else 4.0   # with memories: read g, read and write epsilon
+        achieved = bytes_per_elem * elems / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": "filter_kernel" if st.rows_general == 0 else "general_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": FILTER_TRAFFIC_PER_ROW_CONFIG5 * wl.N if (wl.cid == 5 and not args.d) else None,
-                "algorithmic_bytes": 4 * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
+                "traffic": FILTER_TRAFFIC_PER_ROW_CONFIG5 * wl.N if (wl.cid == 5 and not args.d and not args.ef) else None,
+                "algorithmic_bytes": int(bytes_per_elem) * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
 
     # end to end through tk_step_host: pinned host buffers, copies inside the timed region
     e2e = None
@@ -268,21 +273,27 @@ def main():
         G = bufs[0].cpu().numpy()
         w_cpu = w.cpu().numpy()
         t0 = time.perf_counter()
-        oracle.ref_step(w_cpu, G, wl.K_up, K_down, p.numpy(), wl.alpha, 1, nthreads=threads, want_dense=False)
+        if args.ef:
+            import numpy as np
+            oracle.ref_step_ef(w_cpu, np.zeros_like(G), np.zeros_like(w_cpu), G, wl.K_up, K_down, p.numpy(), wl.alpha, 1,
+                               nthreads=threads)
+        else:
+            oracle.ref_step(w_cpu, G, wl.K_up, K_down, p.numpy(), wl.alpha, 1, nthreads=threads, want_dense=False)
         dt = time.perf_counter() - t0
         cpu = {"value": elems / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": "1 full step of config %d (N=%d rows of d=%d), %.1f s" % (wl.cid, wl.N, wl.d, dt)}
 
     if rank == 0:
         cfg = W.describe(wl)
-        cfg.update({"mode": "bidirectional", "cold_inputs": "each step reads a %d MB gradient tensor (>> L2), "
+        cfg.update({"mode": "bidirectional with error memories" if args.ef else "bidirectional", "cold_inputs": "each step reads a %d MB gradient tensor (>> L2), "
                     "%d distinct tensors cycled" % (4 * elems // 10 ** 6, nbuf),
                     "parallelism": "replicas x%d" % world})
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
-            "hbm_frac_of_8TBps": b_min_bytes(wl, K_down) / (ms_per_step * 1e-3) / NOMINAL_HBM_BPS,
+            "hbm_frac_of_8TBps": (b_min_bytes(wl, K_down) + (8 * elems + 4 * wl.d if args.ef else 0))
+            / (ms_per_step * 1e-3) / NOMINAL_HBM_BPS,
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
             "clocks": sampler.summary(),
             "stats": {"rows_general": st.rows_general, "union_size": st.union_size,

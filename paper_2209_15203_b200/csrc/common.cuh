@@ -56,7 +56,7 @@ constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the mult
 struct RowState {
     u64 lo;          // the row's candidates are exactly the components with ck >= lo
     u32 cand_count;  // how many components have ck >= lo (counted, even beyond capacity)
-    u32 max_key;     // unused by the kernels (kept for layout stability)
+    u32 max_key;     // largest key among them (upper end of the selection's first range)
     u32 out_count;   // entries emitted by the final exact selection
     u32 flags;
     u32 ticket;      // sampling CTAs of this row that have finished

@@ -125,3 +125,12 @@ def test_memory_free_steps_still_work_after_attach():
     assert_values_close(w.cpu().numpy(), ref.w, "memory-free step")
     eps, delta = ctx.tk_ef_state()
     assert not eps.any() and not delta.any()
+
+
+@pytest.mark.parametrize("cid,steps", [(2, 2), (5, 1)])
+def test_full_size_configs_with_memories(cid, steps):
+    import psutil
+    wl = W.workload(cid)
+    if psutil.virtual_memory().available < wl.N * wl.d * 4 * 6 + 16 * wl.d * 8:
+        pytest.skip("not enough host memory for the oracle at this size")
+    run_ef(wl, steps, 1)

@@ -124,6 +124,21 @@ def test_repeatable_bits():
     run_both(G.cpu().numpy(), wl.K_up, x_dev=G)
 
 
+def test_random_shapes_sweep():
+    # many small problems of random shape, half of them tie-heavy: rows, d, K at every alignment
+    rng = np.random.default_rng(2209)
+    mags = np.array([0.0, 1e-3, 0.5, 0.5, 2.0, 7.25, 1e-41], dtype=np.float32)
+    for case in range(60):
+        rows = int(rng.integers(1, 6))
+        d = int(rng.integers(1, 40_000))
+        K = int(rng.integers(1, d + 1)) if case % 3 else int(rng.integers(1, min(d, 50) + 1))
+        if case % 2:
+            x = mags[rng.integers(0, mags.size, (rows, d))] * rng.choice(np.array([-1.0, 1.0], np.float32), (rows, d))
+        else:
+            x = rng.standard_normal((rows, d)) * np.exp(rng.standard_normal((rows, d)) * 2)
+        run_both(x.astype(np.float32), K)
+
+
 def test_argument_errors():
     x = torch.zeros(100, device=DEV)
     with pytest.raises(binding.TkError):
