@@ -216,6 +216,26 @@ int tk_last_downlink(tk_ctx* ctx, int32_t* idx_out_dev, float* val_out_dev, int6
 /* Synchronise the stream and report counters and the sticky device status. */
 int tk_status(tk_ctx* ctx, tk_stats* out);
 
+/*
+ * The paper's per-step diagnostics that do not need the uncompressed aggregate.
+ *   tk_set_diagnostics(ctx, 1)  makes the following steps also accumulate sums of squares
+ *        (one fused multiply-add per value in the streaming pass, fp32 per thread, double across
+ *        threads) and count the non-zeros of the aggregate.  Off by default.
+ *   tk_diagnostics              synchronises and reports, for the last step:
+ */
+typedef struct tk_diag {
+    double nonzero_fraction;        /* nnz(sum_q p_q Top_K(a^q)) / d: the quantity of Fig. 5 / Section 4.2,
+                                       which approaches K_up N / d */
+    double union_fraction;          /* |U| / d (>= nonzero_fraction; they differ when entries cancel) */
+    double compression_factor;      /* K_down / (K_up N): Section 4.2's bound on downlink size vs the aggregate */
+    double one_minus_gamma_up_max;  /* max_q ||Top_K(a^q) - a^q||^2 / ||a^q||^2: the "1 - gamma" estimate of the
+                                       appendix for the uplink compressions (<= (d - K_up)/d by Eq. "topk_bound") */
+    double one_minus_gamma_down;    /* the same for the downlink compression Top_K_down(g); 0 when unidirectional */
+} tk_diag;
+/*   one_minus_gamma_up_host: NULL, or [N] doubles that receive the per-worker values. */
+int tk_set_diagnostics(tk_ctx* ctx, int on);
+int tk_diagnostics(tk_ctx* ctx, tk_diag* out, double* one_minus_gamma_up_host);
+
 /* Record device timestamps around the streaming selection pass of each step (0/1). */
 int tk_set_profile(tk_ctx* ctx, int on);
 

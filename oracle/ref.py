@@ -48,6 +48,8 @@ def _load():
         lib.ref_step.argtypes = [f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
                                  i32p, f32p, f32p, u8p, i32p, f32p, ctypes.c_void_p, ctypes.c_int]
         lib.ref_step.restype = ctypes.c_int
+        lib.ref_lost_energy.argtypes = [f32p, i64, i32p, i64]
+        lib.ref_lost_energy.restype = ctypes.c_double
         lib.ref_step_ef.argtypes = [f32p, f32p, f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
                                     i32p, f32p, i32p, f32p, ctypes.c_void_p, ctypes.c_int]
         lib.ref_step_ef.restype = ctypes.c_int
@@ -187,3 +189,10 @@ def ref_step_ef(w, eps, delta, G, K_up: int, K_down: int, p, alpha: float, mode:
         raise ValueError("ref_step_ef rejected its arguments")
     n = count.value
     return EfResult(w, eps, delta, up_idx, up_val, msg_idx[:n].copy(), msg_val[:n].copy())
+
+
+def ref_lost_energy(x, idx) -> float:
+    """||Top_K(x) - x||^2 / ||x||^2 for the message with indices idx (the appendix's 1 - gamma)."""
+    x = _f32(x).reshape(-1)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    return float(_load().ref_lost_energy(_ptr(x), x.size, _ptr(idx), idx.size))

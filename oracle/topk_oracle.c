@@ -338,3 +338,24 @@ done:
     free(up_idx); free(up_val); free(S); free(touched); free(msg_idx); free(msg_val);
     return rc;
 }
+
+/*
+ * The "1 - gamma" diagnostic of the appendix:  ||Top_K(x) - x||_2^2 / ||x||_2^2  for a
+ * message (idx[K]) taken from x[d], in double precision.  Top_K(x) - x is -x off the message
+ * and 0 on it, so the numerator is the sum of squares of the components NOT sent.
+ * Returns 0 for the zero vector.
+ */
+double ref_lost_energy(const float *x, int64_t d, const int32_t *idx, int64_t K)
+{
+    uint8_t *sent = (uint8_t *)calloc((size_t)d, 1);
+    if (!sent) return -1.0;
+    for (int64_t k = 0; k < K; ++k) sent[idx[k]] = 1;
+    double lost = 0.0, total = 0.0;
+    for (int64_t j = 0; j < d; ++j) {
+        double v = (double)x[j];
+        total += v * v;
+        if (!sent[j]) lost += v * v;
+    }
+    free(sent);
+    return total > 0.0 ? lost / total : 0.0;
+}

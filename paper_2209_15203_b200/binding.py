@@ -21,7 +21,7 @@ TK_MODE_BIDIR = 1
 TK_MODE_EF = 2
 
 EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
-           "tk_ef_attach", "tk_ef_state", "tk_set_kdown",
+           "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
            "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
@@ -37,6 +37,12 @@ class tk_stats(ctypes.Structure):
                 ("union_size", ctypes.c_int64), ("downlink_count", ctypes.c_int64),
                 ("cand_min", ctypes.c_int64), ("cand_max", ctypes.c_int64),
                 ("select_ms_sum", ctypes.c_float), ("select_samples", ctypes.c_int32)]
+
+
+class tk_diag(ctypes.Structure):
+    _fields_ = [("nonzero_fraction", ctypes.c_double), ("union_fraction", ctypes.c_double),
+                ("compression_factor", ctypes.c_double), ("one_minus_gamma_up_max", ctypes.c_double),
+                ("one_minus_gamma_down", ctypes.c_double)]
 
 
 _lib = None
@@ -75,6 +81,10 @@ def load(build_if_missing: bool = True):
     lib.tk_ef_attach.restype = ctypes.c_int
     lib.tk_ef_state.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.tk_ef_state.restype = ctypes.c_int
+    lib.tk_set_diagnostics.argtypes = [vp, ctypes.c_int]
+    lib.tk_set_diagnostics.restype = ctypes.c_int
+    lib.tk_diagnostics.argtypes = [vp, ctypes.POINTER(tk_diag), ctypes.POINTER(ctypes.c_double)]
+    lib.tk_diagnostics.restype = ctypes.c_int
     lib.tk_set_kdown.argtypes = [vp, i64]
     lib.tk_last_uplink.argtypes = [vp, vp, vp]
     lib.tk_last_aggregate.argtypes = [vp, vp, vp, ctypes.POINTER(i64)]
@@ -186,6 +196,16 @@ class Context:
         flat = self.ef_memory.view(torch.float32)
         eo, do = (e.value - base) // 4, (dl.value - base) // 4
         return flat[eo:eo + self.N * self.d].view(self.N, self.d), flat[do:do + self.d]
+
+    def tk_set_diagnostics(self, on: bool) -> None:
+        _check(load().tk_set_diagnostics(self._h, 1 if on else 0), "tk_set_diagnostics")
+
+    def tk_diagnostics(self):
+        """(tk_diag, per-worker 1 - gamma list) of the last step."""
+        out = tk_diag()
+        per = (ctypes.c_double * self.N)()
+        _check(load().tk_diagnostics(self._h, ctypes.byref(out), per), "tk_diagnostics")
+        return out, list(per)
 
     def tk_set_kdown(self, K_down: int) -> None:
         _check(load().tk_set_kdown(self._h, K_down), "tk_set_kdown")

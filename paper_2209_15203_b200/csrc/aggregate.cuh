@@ -21,7 +21,8 @@ namespace tk {
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
                   u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
-                  uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d) {
+                  uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
+                  int stats) {
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
     u32 j = 0;
@@ -70,6 +71,11 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     if (owner) {
         u32 slot = sh_base + incl - 1;
         if (slot < ucap) U[slot] = make_uint2(j, bits);
+    }
+    if (stats) {  // diagnostics: non-zeros of the aggregate (Section 4.2) and its squared norm
+        u32 nz = __reduce_add_sync(0xffffffffu, (owner && key_of(bits) != 0) ? 1u : 0u);
+        if (lane_id() == 0 && nz) atomicAdd(&uni->nnz, nz);
+        warp_add_double(&uni->sum_sq, owner ? (double)acc * (double)acc : 0.0);
     }
 }
 

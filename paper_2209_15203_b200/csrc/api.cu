@@ -185,6 +185,7 @@ struct tk_ctx {
     u32 ucap = 0;
     // host state
     int force_general = 0;
+    int diagnostics = 0;
     int profile = 0;
     int last_mode = -1;
     int64_t last_kdown = 0;
@@ -279,9 +280,9 @@ int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, siz
 
 // One long list selected by the whole grid (cooperative launch).
 int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap, RowState* rs, u32 K, uint2* out,
-                       ApplyArgs apply, Ctrl* ctrl, u32* ghist) {
+                       ApplyArgs apply, Ctrl* ctrl, u32* ghist, bool stats) {
     size_t stride = cap;
-    LinkArgs nolink = {nullptr, nullptr, 0, 0};
+    LinkArgs nolink = {nullptr, nullptr, 0, 0, nullptr, 0, stats ? 1 : 0};
     void* args[] = {(void*)&list, (void*)&stride, (void*)&cap, (void*)&rs,  (void*)&K,    (void*)&out,
                     (void*)&stride, (void*)&apply, (void*)&nolink, (void*)&ctrl, (void*)&ghist};
     if (cudaLaunchCooperativeKernel((void*)select_kernel<true>, dim3(ctas), dim3(kSelectThreads), args, 0, stream) !=
@@ -301,7 +302,7 @@ int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap
 int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
                Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches,
                RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0},
-               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}) {
+               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}, bool stats = false) {
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
@@ -361,12 +362,15 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             u32 parts = 1;
             if (tiles >= 4 * resident) parts = (u32)(nr < kFilterPartitions ? nr : kFilterPartitions);
             u32 cpp = grid / parts;
-            if (fused)
-                filter_kernel<true><<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, tprf, parts, cpp,
-                                                                                              rs, cand, b.cap, efb);
+            size_t shm = (size_t)nr * sizeof(u64);
+            if (fused && stats)
+                filter_kernel<true, true><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
+            else if (fused)
+                filter_kernel<true, false><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
+            else if (stats)
+                filter_kernel<false, true><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
             else
-                filter_kernel<false><<<grid, kFilterThreads, (size_t)nr * sizeof(u64), stream>>>(xb, nr, d, tprf, parts, cpp,
-                                                                                               rs, cand, b.cap, efb);
+                filter_kernel<false, false><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
             TK_LAUNCH_CHECK();
             if (fused) xb = efb.eps;  // the compensated vector now sits in eps: what a re-filter must read
             if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
@@ -378,8 +382,9 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         }
         {
             u32 Ku = (u32)K, tpr = b.tpr_general, cap = b.cap;
+            int st = stats ? 1 : 0;
             void* args[] = {(void*)&xb, (void*)&nr, (void*)&d, (void*)&Ku, (void*)&tpr, (void*)&cap,
-                            (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl};
+                            (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl, (void*)&st};
             // without a prediction the multi-pass kernel is the streaming pass that gets timed
             if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kGeneralThreads), args,
@@ -393,6 +398,7 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         int64_t expect = predict ? 2 * K : (int64_t)b.cap;
         LinkArgs lk = link;
         lk.row_base = (u32)r0;
+        lk.stats = stats ? 1 : 0;
         if (lk.zero_src) lk.zero_src += (size_t)r0 * lk.zero_stride;
         rc = launch_select(stream, nr, cluster_size_for(expect, nr, di->sms), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, apply,
                            lk, ctrl);
@@ -511,10 +517,11 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     // the first kernel of the selection also resets the state of the union / downlink selection
     // ... and its last kernel threads every uplink entry onto its coordinate's chain (and, with
     // error memories, zeroes the sent entries in eps)
-    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d};
+    const bool diag = c->diagnostics != 0;
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0};
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
     int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
-                        &c->launches, c->uni, link, ef);
+                        &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
     if (rc != TK_OK) return rc;
     // with memories the step size is already inside the messages
     const float scale = with_ef ? 1.0f : alpha;
@@ -522,16 +529,16 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     u32 blocks = (total + 255) / 256;
     agg_reduce_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->uni, c->U,
                                              c->ucap, w_dev, scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : nullptr,
-                                             c->ctrl, (u32)c->d);
+                                             c->ctrl, (u32)c->d, diag ? 1 : 0);
     TK_LAUNCH_CHECK();
     c->launches += 1;
     if (bidir && with_ef) {
         // Algorithm 2 with the server memory: delta now holds g = sum + delta everywhere; take
         // Top_K_down out of it (delta <- g - Top_K(g)) and apply it (w <- w - Top_K(g))
-        LinkArgs zero = {nullptr, nullptr, 0, 0, c->delta, (size_t)c->d};
+        LinkArgs zero = {nullptr, nullptr, 0, 0, c->delta, (size_t)c->d, 0};
         ApplyArgs ap = {w_dev, 1.0f};
         rc = run_select(s, c->delta, 1, c->d, c->K_down, c->down, c->ctrl, c->force_general != 0, nullptr, nullptr,
-                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap);
+                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag);
         if (rc != TK_OK) return rc;
     } else if (bidir) {
         ApplyArgs ap = {w_dev, alpha};
@@ -542,7 +549,7 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
         int ctas = (int)((c->ucap + 4095) / 4096);
         if (ctas > di->select_grid) ctas = di->select_grid;
         if (ctas < 1) ctas = 1;
-        rc = launch_select_grid(s, ctas, c->U, c->ucap, c->uni, (u32)c->K_down, c->sel, ap, c->ctrl, c->ghist);
+        rc = launch_select_grid(s, ctas, c->U, c->ucap, c->uni, (u32)c->K_down, c->sel, ap, c->ctrl, c->ghist, diag);
         if (rc != TK_OK) return rc;
         c->launches += 1;
     }
@@ -791,6 +798,53 @@ int tk_set_profile(tk_ctx* c, int on) {
     }
     c->profile = on ? 1 : 0;
     c->ev_used = 0;
+    return TK_OK;
+}
+
+int tk_set_diagnostics(tk_ctx* c, int on) {
+    if (!c) return TK_ERR_INVALID;
+    c->diagnostics = on ? 1 : 0;
+    return TK_OK;
+}
+
+int tk_diagnostics(tk_ctx* c, tk_diag* out, double* one_minus_gamma_up_host) {
+    if (!c || !out || c->last_mode < 0 || !c->diagnostics) return TK_ERR_INVALID;
+    memset(out, 0, sizeof *out);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    RowState u, dn;
+    memset(&dn, 0, sizeof dn);
+    RowState* rows = new (std::nothrow) RowState[c->N];
+    if (!rows) return TK_ERR_ALLOC;
+    const bool ef_bidir = c->last_mode == (TK_MODE_BIDIR | TK_MODE_EF);
+    bool ok = cudaMemcpy(&u, c->uni, sizeof u, cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemcpy(rows, c->up.rs, (size_t)c->N * sizeof(RowState), cudaMemcpyDeviceToHost) == cudaSuccess &&
+              (!ef_bidir || cudaMemcpy(&dn, c->down.rs, sizeof dn, cudaMemcpyDeviceToHost) == cudaSuccess);
+    if (!ok) {
+        delete[] rows;
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    auto lost = [](double total, double kept) {   // ||Top_K(x) - x||^2 / ||x||^2
+        if (!(total > 0.0)) return 0.0;
+        double v = 1.0 - kept / total;
+        return v < 0.0 ? 0.0 : v;
+    };
+    double worst = 0.0;
+    for (int q = 0; q < c->N; ++q) {
+        double v = lost(rows[q].sum_sq, rows[q].sel_sq);
+        if (one_minus_gamma_up_host) one_minus_gamma_up_host[q] = v;
+        if (v > worst) worst = v;
+    }
+    delete[] rows;
+    out->one_minus_gamma_up_max = worst;
+    out->union_fraction = (double)u.cand_count / (double)c->d;
+    out->nonzero_fraction = (double)u.nnz / (double)c->d;
+    out->compression_factor = (double)c->last_kdown / ((double)c->K_up * (double)c->N);
+    if (ef_bidir) out->one_minus_gamma_down = lost(dn.sum_sq, dn.sel_sq);
+    else if (c->last_mode & TK_MODE_BIDIR) out->one_minus_gamma_down = lost(u.sum_sq, u.sel_sq);
     return TK_OK;
 }
 

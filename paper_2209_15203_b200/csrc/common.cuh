@@ -51,6 +51,7 @@ constexpr int kFilterPartitions = 8;   // the filter grid splits the tile space 
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path
+constexpr u32 kRowNoFilter = 2u;       // RowState.flags: no filter pass has read this row
 
 // Per-row state of one batched selection.  Lives in global memory.
 struct RowState {
@@ -64,6 +65,11 @@ struct RowState {
     u64 g_lo;        // multi-pass path: known leading bits of the K-th composite key
     u32 g_need;      // multi-pass path: entries still to take inside the current bucket
     u32 g_level;
+    // diagnostics (filled only when asked for)
+    double sum_sq;   // sum of squares of the whole vector
+    double sel_sq;   // sum of squares of the emitted entries
+    u32 nnz;         // union list: entries whose value is not zero
+    u32 pad;
 };
 
 // Step-wide control block.
@@ -113,6 +119,18 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 }
 
 __device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31; }
+
+// *dst += sum over the warp of v, accumulated in double.  All lanes call.
+__device__ __forceinline__ void warp_add_double(double* dst, double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane_id() == 0 && v != 0.0) atomicAdd(dst, v);
+}
+
+__device__ __forceinline__ float sq4(uint4 v, float acc) {
+    float a = __uint_as_float(v.x), b = __uint_as_float(v.y), c = __uint_as_float(v.z), e = __uint_as_float(v.w);
+    return fmaf(a, a, fmaf(b, b, fmaf(c, c, fmaf(e, e, acc))));
+}
 
 // Append the lanes with `pred` to a list whose fill counter is *counter.
 // Every lane of the warp must call.  The counter always advances by the number

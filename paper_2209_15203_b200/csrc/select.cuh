@@ -46,6 +46,9 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->flags = flags;
     r->ticket = 0;
     r->g_active = 0;
+    r->sum_sq = 0.0;
+    r->sel_sq = 0.0;
+    r->nnz = 0;
 }
 
 template <bool kEF>
@@ -148,7 +151,7 @@ __global__ void __launch_bounds__(256) compensate_kernel(float* eps, const float
 // No prediction: mark every row for the multi-pass path.
 __global__ void reset_rows_kernel(RowState* rs, int rows, RowState* also_reset) {
     int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r < rows) reset_state(rs + r, ~0ull, kRowGeneral);
+    if (r < rows) reset_state(rs + r, ~0ull, kRowGeneral | kRowNoFilter);
     if (also_reset && r == 0) reset_state(also_reset, 0ull, 0u);
 }
 
@@ -279,10 +282,11 @@ __device__ __forceinline__ bool may_hit(uint4 v, float thr) {
 // With kEF the row's memory `erow` is read as well, the compensated vector a = eps + alpha*g
 // is what gets filtered, and it is written back to the memory (the entries sent later are
 // zeroed there by the selection's emission: eps <- a - Top_K(a)).
-template <int THREADS, int UNROLL, bool kEF>
+// With kStats the squares of all values of the tile are added to `sq` (per thread, fp32).
+template <int THREADS, int UNROLL, bool kEF, bool kStats>
 __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
-                                            RowState* rs, uint2* cand, u32 cap, float* erow = nullptr,
-                                            float alpha = 0.0f) {
+                                            RowState* rs, uint2* cand, u32 cap, float* erow, float alpha,
+                                            float& sq) {
     const u32 tk = (u32)(lo >> 32);
     const float thr = __uint_as_float(tk);
     const u32 j0 = tile * (THREADS * UNROLL) + threadIdx.x;
@@ -318,6 +322,10 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
             else v[u] = make_uint4(0, 0, 0, 0);
         }
     }
+    if (kStats) {  // lanes outside the row hold zeros
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) sq = sq4(v[u], sq);
+    }
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
         bool hit = inb[u] && may_hit(v[u], thr);
@@ -344,6 +352,7 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
             bits = compensated(bits, __float_as_uint(erow[idx]), alpha);
             erow[idx] = __uint_as_float(bits);
         }
+        if (kStats && live) sq = fmaf(__uint_as_float(bits), __uint_as_float(bits), sq);
         consider(live, idx, bits, lo, st, rs, cand, cap);
     }
 }
@@ -353,7 +362,7 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
 // range every CTA would visit every row, and each change of row costs a flush of the
 // staged candidates (a global atomic round trip); with one range per CTA a CTA that
 // lands in a layer full of candidates would finish late.
-template <bool kEF>
+template <bool kEF, bool kStats>
 __global__ void __launch_bounds__(kFilterThreads, kFilterCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 parts, u32 cpp,
               RowState* rs, uint2* cand, u32 cap, EfArgs ef) {
@@ -375,20 +384,28 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
     u64 lo = 0;
     int row = (int)(t / tpr);
     u32 tile = (u32)(t - (u64)row * tpr);
+    float sq = 0.0f;
     for (; t < t_end; t += cpp) {
         if (row != cur) {
-            if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
+            if (cur >= 0) {
+                stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
+                if (kStats) { warp_add_double(&rs[cur].sum_sq, (double)sq); sq = 0.0f; }
+            }
             cur = row;
             g = row_geom(x, row, d);
             lo = sh_lo[row];
         }
         if (tile * (u32)(kFilterThreads * kUnroll) < g.nv || tile == 0)
-            filter_tile<kFilterThreads, kUnroll, kEF>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap,
-                                                      kEF ? ef.eps + (size_t)row * (size_t)d : nullptr, ef.alpha);
+            filter_tile<kFilterThreads, kUnroll, kEF, kStats>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap,
+                                                              kEF ? ef.eps + (size_t)row * (size_t)d : nullptr, ef.alpha,
+                                                              sq);
         tile += cpp;
         while (tile >= tpr) { tile -= tpr; ++row; }
     }
-    if (cur >= 0) stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
+    if (cur >= 0) {
+        stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
+        if (kStats) warp_add_double(&rs[cur].sum_sq, (double)sq);
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -415,8 +432,9 @@ __device__ __forceinline__ void hist_component(bool live, u32 idx, u32 bits, int
     atomicAdd(&sh_hist[(u32)(ck >> shift) & ((1u << nbits) - 1u)], 1u);
 }
 
+// `sq`, when given, also receives the squares of all values of the tile (diagnostics).
 __device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level, u64 lo,
-                                          u32* sh_hist) {
+                                          u32* sh_hist, float* sq) {
     const int shift = kLevelShift[level], nbits = kLevelBits[level];
     const u32 j0 = tile * kGeneralTileVecs + threadIdx.x;
 #pragma unroll
@@ -425,6 +443,7 @@ __device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level,
         if (j < g.nv) {
             uint4 v = ld_stream(g.vec + j);
             u32 i0 = g.head + 4u * j;
+            if (sq) *sq = sq4(v, *sq);
             hist_component(true, i0 + 0, v.x, level, shift, nbits, lo, sh_hist);
             hist_component(true, i0 + 1, v.y, level, shift, nbits, lo, sh_hist);
             hist_component(true, i0 + 2, v.z, level, shift, nbits, lo, sh_hist);
@@ -438,6 +457,7 @@ __device__ __forceinline__ void hist_tile(const RowGeom& g, u32 tile, int level,
         if (lane < g.head) { live = true; idx = lane; }
         else if (lane >= 8 && lane - 8 < g.tail) { live = true; idx = g.head + 4u * g.nv + (lane - 8); }
         u32 bits = live ? __float_as_uint(__ldg(g.base + idx)) : 0u;
+        if (sq && live) *sq = fmaf(__uint_as_float(bits), __uint_as_float(bits), *sq);
         hist_component(live, idx, bits, level, shift, nbits, lo, sh_hist);
     }
 }
@@ -464,7 +484,7 @@ __device__ __forceinline__ int build_row_list(int rows, unsigned short* sh_list,
 
 __global__ void __launch_bounds__(kGeneralThreads)
 general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr, u32 cap,
-               RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl) {
+               RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl, int stats) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ unsigned short sh_list[kMaxRowsPerLaunch];
     __shared__ u32 sh_scratch[33];
@@ -511,6 +531,8 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
             int cur = -1, row = 0, level = 0;
             u64 lo = 0;
             RowGeom g;
+            float sq = 0.0f;
+            bool want_sq = false;  // the first full pass over a row no filter pass has read also sums its squares
             for (u64 t = t0; t < t1; ++t) {
                 int li = (int)(t / tpr);
                 u32 tile = (u32)(t - (u64)li * tpr);
@@ -519,6 +541,8 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
                         __syncthreads();
                         for (int b = threadIdx.x; b < kHistBins; b += blockDim.x)
                             if (sh_hist[b]) atomicAdd(&hist[(size_t)row * kHistBins + b], sh_hist[b]);
+                        if (want_sq) warp_add_double(&rs[row].sum_sq, (double)sq);
+                        sq = 0.0f;
                     }
                     __syncthreads();
                     cur = li;
@@ -526,16 +550,18 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
                     g = row_geom(x, row, d);
                     lo = rs[row].g_lo;
                     level = (int)rs[row].g_level;
+                    want_sq = stats && level == 0 && (rs[row].flags & kRowNoFilter) != 0;
                     for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
                     __syncthreads();
                 }
                 if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
-                hist_tile(g, tile, level, lo, sh_hist);
+                hist_tile(g, tile, level, lo, sh_hist, want_sq ? &sq : nullptr);
             }
             if (cur >= 0) {
                 __syncthreads();
                 for (int b = threadIdx.x; b < kHistBins; b += blockDim.x)
                     if (sh_hist[b]) atomicAdd(&hist[(size_t)row * kHistBins + b], sh_hist[b]);
+                if (want_sq) warp_add_double(&rs[row].sum_sq, (double)sq);
             }
         }
         grid.sync();
@@ -599,7 +625,11 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
             lo = rs[row].lo;
         }
         if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
-        filter_tile<kGeneralThreads, kStreamUnroll, false>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap);
+        {
+            float unused = 0.0f;
+            filter_tile<kGeneralThreads, kStreamUnroll, false, false>(g, tile, lo, st, rs + row, cand + (size_t)row * cap,
+                                                                      cap, nullptr, 0.0f, unused);
+        }
     }
     if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
 }
@@ -624,6 +654,7 @@ struct LinkArgs {
     // (eps <- a - Top_K(a), delta <- g - Top_K(g): second worker / server line of Algorithm 1/2).
     float* zero_src;
     size_t zero_stride;
+    int stats;  // diagnostics: add the squares of the emitted values to RowState.sel_sq
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
@@ -769,6 +800,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
 
     // emission: every entry with ck >= T, exactly Keff of them; one counter update per warp
     uint2* orow = out + (size_t)row * out_stride;
+    double sel_sq = 0.0;
     u32 mine = 0;
 #pragma unroll
     for (int k = 0; k < kSelectRegs; ++k) mine += eck[k] >= T ? 1u : 0u;
@@ -793,6 +825,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                 u32 idx = 0xffffffffu - (u32)eck[k];
                 u32 bits = (u32)(eck[k] >> 32) | (((esign >> k) & 1u) << 31);
                 emit_entry(row, slot, Keff, idx, bits, orow, out_stride, apply, link, ctrl);
+                if (link.stats) sel_sq += (double)__uint_as_float(bits) * (double)__uint_as_float(bits);
                 ++slot;
             }
         }
@@ -811,9 +844,13 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         int leader = __ffs(m) - 1;
         if ((int)lane == leader) base = atomicAdd(&r->out_count, (u32)__popc(m));
         base = __shfl_sync(0xffffffffu, base, leader);
-        if (pred) emit_entry(row, base + (u32)__popc(m & ((1u << lane) - 1u)), Keff, e.x, e.y, orow, out_stride,
-                             apply, link, ctrl);
+        if (pred) {
+            emit_entry(row, base + (u32)__popc(m & ((1u << lane) - 1u)), Keff, e.x, e.y, orow, out_stride, apply, link,
+                       ctrl);
+            if (link.stats) sel_sq += (double)__uint_as_float(e.y) * (double)__uint_as_float(e.y);
+        }
     }
+    if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
 }
 
 }  // namespace tk

@@ -168,6 +168,47 @@ def test_same_input_twice_gives_identical_bytes():
     assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2].view(torch.int32), outs[1][2].view(torch.int32))
 
 
+def test_diagnostics_match_the_oracle():
+    # Section 4.2's non-zero fraction and the appendix's 1 - gamma, memory-free and with memories
+    for wl, ef in ((W.workload(4, d=600_000, N=6), False), (W.workload(2, d=500_000, N=4), True),
+                   (W.workload(1, d=30_000), False)):
+        p = W.make_p(wl)
+        K_down = wl.K_down[0]
+        ctx = make_ctx(wl, K_down)
+        ctx.tk_set_diagnostics(True)
+        if ef:
+            ctx.tk_ef_attach()
+        w = W.make_w(wl, DEV)
+        w_ref = w.cpu().numpy()
+        eps = np.zeros((wl.N, wl.d), np.float32)
+        delta = np.zeros(wl.d, np.float32)
+        for s in range(2):
+            G = W.make_grads(wl, s, DEV)
+            Gh = G.cpu().numpy()
+            ctx.tk_step(w, G, wl.alpha, 1 | (binding.TK_MODE_EF if ef else 0))
+            diag, per = ctx.tk_diagnostics()
+            if ef:
+                a = (eps + np.float32(wl.alpha) * Gh).astype(np.float32)
+                ref = oracle.ref_step_ef(w_ref, eps, delta, Gh, wl.K_up, K_down, p.numpy(), wl.alpha, 1)
+                S, _ = oracle.ref_aggregate(ref.up_idx, ref.up_val, p.numpy(), wl.d)
+                g = (S + delta).astype(np.float32)
+                eps, delta = ref.eps, ref.delta
+            else:
+                a = Gh
+                ref = oracle.ref_step(w_ref, Gh, wl.K_up, K_down, p.numpy(), wl.alpha, 1)
+                S = g = ref.A
+            w_ref = ref.w
+            want = [oracle.ref_lost_energy(a[q], ref.up_idx[q]) for q in range(wl.N)]
+            assert np.allclose(per, want, rtol=0, atol=2e-5)
+            assert abs(diag.one_minus_gamma_up_max - max(want)) < 2e-5
+            assert diag.one_minus_gamma_up_max <= (wl.d - wl.K_up) / wl.d + 2e-5     # Eq. "topk_bound"
+            assert abs(diag.one_minus_gamma_down - oracle.ref_lost_energy(g, ref.msg_idx)) < 2e-5
+            assert diag.nonzero_fraction == np.count_nonzero(S) / wl.d
+            assert diag.nonzero_fraction <= diag.union_fraction <= wl.N * wl.K_up / wl.d
+            assert diag.compression_factor == K_down / (wl.K_up * wl.N)
+        ctx.close()
+
+
 def test_bad_arguments_are_rejected():
     wl = W.workload(1, d=1000)
     ctx = make_ctx(wl, 10)

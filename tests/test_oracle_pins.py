@@ -244,3 +244,28 @@ def test_rejects_bad_arguments():
         oracle.ref_topk(np.zeros(4, np.float32), 5)
     with pytest.raises(ValueError):
         oracle.ref_topk(np.zeros(4, np.float32), 0)
+
+
+def test_lost_energy_closed_forms_and_bound():
+    # constant vector: Top_K keeps K of d equal squares, so the bound of Eq. "topk_bound" is attained
+    d, K = 1000, 37
+    x = np.full(d, -1.5, np.float32)
+    idx, _ = oracle.ref_topk(x, K)
+    assert abs(oracle.ref_lost_energy(x, idx) - (d - K) / d) < 1e-15
+    # at most K non-zeros: nothing is lost; zero vector: defined as 0
+    y = np.zeros(d, np.float32)
+    y[[3, 500, 999]] = [2.0, -7.0, 0.5]
+    idx, _ = oracle.ref_topk(y, 3)
+    assert oracle.ref_lost_energy(y, idx) == 0.0
+    assert oracle.ref_lost_energy(np.zeros(d, np.float32), idx) == 0.0
+    # one dominant component: what is lost is the rest, by hand
+    z = np.array([3.0, 4.0, 12.0], np.float32)
+    idx, _ = oracle.ref_topk(z, 1)
+    assert abs(oracle.ref_lost_energy(z, idx) - 25.0 / 169.0) < 1e-15
+    # random data: below the bound, and scale-free
+    rng = np.random.default_rng(21)
+    r = rng.standard_t(3, 5000).astype(np.float32)
+    idx, _ = oracle.ref_topk(r, 50)
+    v = oracle.ref_lost_energy(r, idx)
+    assert 0 < v <= (5000 - 50) / 5000
+    assert abs(oracle.ref_lost_energy((r * np.float32(0.25)).astype(np.float32), idx) - v) < 1e-12
