@@ -164,6 +164,8 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the vector length d (smaller case for profiling)")
     ap.add_argument("--ef", action="store_true", help="keep the error memories (Algorithm 2 as printed): "
                     "12 bytes per gradient value instead of 4")
+    ap.add_argument("--sharded", action="store_true", help="with --gpus N > 1: shard the N workers over the ranks "
+                    "(one all-gather of the messages per step) instead of running independent replicas")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -178,7 +180,7 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2209_15203_b200 import binding, replicas
+    from paper_2209_15203_b200 import binding, replicas, sharding
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -206,8 +208,20 @@ def main():
         replicas.barrier()
         torch.cuda.synchronize()
 
+    if args.sharded:
+        # strong scaling: this rank keeps (and steps) its own workers' rows only
+        row0, nrows = sharding.row_range(wl.N, rank, world)
+        bufs = [b[row0:row0 + nrows].clone() for b in bufs]
+        torch.cuda.empty_cache()
+
+        def step(g):
+            sharding.sharded_step(ctx, w, g, wl.alpha, mode)
+    else:
+        def step(g):
+            ctx.tk_step(w, g, wl.alpha, mode)
+
     for s in range(warmup):
-        ctx.tk_step(w, bufs[s % nbuf], wl.alpha, mode)
+        step(bufs[s % nbuf])
     st = ctx.tk_status()
     ctx.tk_set_profile(True)
 
@@ -218,7 +232,7 @@ def main():
     sampler.start()
     ev0.record()
     for s in range(args.steps):
-        ctx.tk_step(w, bufs[s % nbuf], wl.alpha, mode)
+        step(bufs[s % nbuf])
     ev1.record()
     barrier()
     sampler.stop_flag = True
@@ -230,6 +244,8 @@ def main():
 
     elems = wl.N * wl.d
     value, ms_max = replicas.whole_job_throughput(ms, elems, args.steps, dev)
+    if args.sharded:
+        value /= world          # one job of N*d values per step, not one per rank
     ms_per_step = ms_max / args.steps
 
     # roofline of the dominant kernel (the streaming selection pass)
@@ -238,15 +254,16 @@ def main():
     if st.select_samples > 0 and st.select_ms_sum > 0:
         k_ms = st.select_ms_sum / st.select_samples
         bytes_per_elem = 12.0 if args.ef else 4.0   # with memories: read g, read and write epsilon
-        achieved = bytes_per_elem * elems / (k_ms * 1e-3) / 1e9
+        elems_rank = (elems // world) if args.sharded else elems     # what one launch on this rank reads
+        achieved = bytes_per_elem * elems_rank / (k_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": "filter_kernel" if st.rows_general == 0 else "general_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind,
                 "traffic": FILTER_TRAFFIC_PER_ROW_CONFIG5 * wl.N if (wl.cid == 5 and not args.d and not args.ef) else None,
-                "algorithmic_bytes": int(bytes_per_elem) * elems, "kernel_ms": k_ms, "launches_timed": st.select_samples}
+                "algorithmic_bytes": int(bytes_per_elem) * elems_rank, "kernel_ms": k_ms, "launches_timed": st.select_samples}
 
     # end to end through tk_step_host: pinned host buffers, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.sharded:
         g_host = torch.empty((wl.N, wl.d), dtype=torch.float32, pin_memory=True)
         g_host.copy_(bufs[0])
         w_host = torch.empty(wl.d, dtype=torch.float32, pin_memory=True)
@@ -267,7 +284,7 @@ def main():
 
     # the CPU oracle on this host's cores: one full step of the same workload (rank 0, single GPU only)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.sharded:
         import oracle
         threads = min(wl.N, oracle.ref.default_threads())
         G = bufs[0].cpu().numpy()
@@ -287,10 +304,12 @@ def main():
         cfg = W.describe(wl)
         cfg.update({"mode": "bidirectional with error memories" if args.ef else "bidirectional", "cold_inputs": "each step reads a %d MB gradient tensor (>> L2), "
                     "%d distinct tensors cycled" % (4 * elems // 10 ** 6, nbuf),
-                    "parallelism": "replicas x%d" % world})
+                    "parallelism": ("workers sharded over %d ranks, one all-gather per step" if args.sharded
+                                    else "replicas x%d") % world})
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "strong" if args.sharded else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
             "hbm_frac_of_8TBps": (b_min_bytes(wl, K_down) + (8 * elems + 4 * wl.d if args.ef else 0))
             / (ms_per_step * 1e-3) / NOMINAL_HBM_BPS,

@@ -110,6 +110,28 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down,
 int tk_step(tk_ctx* ctx, float* w_dev, const float* grads_dev, float alpha, int mode);
 
 /*
+ * The same iteration with the workers spread over several GPUs (one process per GPU): the
+ * uplink SEND / RECV of Algorithm 1/2 becomes one all-gather of the N messages.  Every process
+ * creates its context with the FULL N and p, holds the gradients of its own rows only, and does
+ *   tk_step_uplink(ctx, grads_local, row0, rows, alpha, mode)
+ *        stage 1 for workers row0 .. row0+rows-1 (grads_local_dev: [rows][d]); their messages
+ *        land in rows row0.. of the message buffer (with TK_MODE_EF only those rows' memories
+ *        are used and updated)
+ *   tk_messages(ctx, &msgs, &bytes_per_row)
+ *        the message buffer: [N] rows of K_up entries of 8 bytes (int32 index, fp32 value), in
+ *        the context's workspace.  The caller gathers it across processes so that every process
+ *        holds all N rows (e.g. an in-place NCCL all-gather when every rank owns N/world rows).
+ *   tk_step_server(ctx, w, alpha, mode)
+ *        stages 2-4 on the gathered messages.  Every process computes the same sums in the same
+ *        worker order, so the replicas of w (and of delta) stay bit-identical.
+ * All three are asynchronous on the context's stream; order the exchange after it.
+ * tk_step is tk_step_uplink over all rows followed by tk_step_server, fused.
+ */
+int tk_step_uplink(tk_ctx* ctx, const float* grads_local_dev, int32_t row0, int32_t rows, float alpha, int mode);
+int tk_messages(tk_ctx* ctx, void** msgs_dev, size_t* bytes_per_row);
+int tk_step_server(tk_ctx* ctx, float* w_dev, float alpha, int mode);
+
+/*
  * The same iteration for callers whose data lives in host memory: copies
  * grads_host ([N][d]) and w_host ([d]) to staging buffers the context allocates
  * on first use (cudaMalloc, 4*(N+1)*d bytes), runs tk_step, copies w back and

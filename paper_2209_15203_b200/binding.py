@@ -20,7 +20,7 @@ TK_MODE_UNI = 0
 TK_MODE_BIDIR = 1
 TK_MODE_EF = 2
 
-EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
+EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
            "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
            "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
@@ -72,6 +72,12 @@ def load(build_if_missing: bool = True):
     lib.tk_init.argtypes = [ctypes.POINTER(vp), i64, i32, i64, i64, vp, vp, ctypes.c_size_t, vp]
     lib.tk_step.argtypes = [vp, vp, vp, f32, ctypes.c_int]
     lib.tk_step_host.argtypes = [vp, vp, vp, f32, ctypes.c_int]
+    lib.tk_step_uplink.argtypes = [vp, vp, i32, i32, f32, ctypes.c_int]
+    lib.tk_step_uplink.restype = ctypes.c_int
+    lib.tk_messages.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
+    lib.tk_messages.restype = ctypes.c_int
+    lib.tk_step_server.argtypes = [vp, vp, f32, ctypes.c_int]
+    lib.tk_step_server.restype = ctypes.c_int
     lib.tk_topk.argtypes = [vp, vp, i32, i64, i64, vp, vp]
     lib.tk_topk_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, vp]
     lib.tk_topk_noalloc.restype = ctypes.c_int
@@ -163,6 +169,25 @@ class Context:
     def tk_step(self, w: torch.Tensor, grads: torch.Tensor, alpha: float, mode: int) -> None:
         assert w.numel() == self.d and grads.numel() == self.N * self.d
         _check(load().tk_step(self._h, _dev(w, torch.float32), _dev(grads, torch.float32), alpha, mode), "tk_step")
+        self.last_mode = mode
+
+    def tk_step_uplink(self, grads_local: torch.Tensor, row0: int, alpha: float, mode: int) -> None:
+        rows = grads_local.numel() // self.d
+        assert grads_local.numel() == rows * self.d
+        _check(load().tk_step_uplink(self._h, _dev(grads_local, torch.float32), row0, rows, alpha, mode),
+               "tk_step_uplink")
+
+    def tk_messages(self) -> torch.Tensor:
+        """The message buffer as an int64 view [N][K_up] of the workspace (one 8-byte entry =
+        int32 index in the low half, fp32 bits in the high half), for the all-gather."""
+        ptr, per_row = ctypes.c_void_p(), ctypes.c_size_t()
+        _check(load().tk_messages(self._h, ctypes.byref(ptr), ctypes.byref(per_row)), "tk_messages")
+        off = (ptr.value - self.workspace.data_ptr()) // 8
+        return self.workspace.view(torch.int64)[off:off + self.N * self.K_up].view(self.N, self.K_up)
+
+    def tk_step_server(self, w: torch.Tensor, alpha: float, mode: int) -> None:
+        assert w.numel() == self.d
+        _check(load().tk_step_server(self._h, _dev(w, torch.float32), alpha, mode), "tk_step_server")
         self.last_mode = mode
 
     def tk_step_host(self, w_host: torch.Tensor, grads_host: torch.Tensor, alpha: float, mode: int) -> None:

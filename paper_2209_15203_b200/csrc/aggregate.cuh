@@ -18,6 +18,22 @@
 
 namespace tk {
 
+// Threads every entry of a gathered message buffer onto its coordinate's chain — what the
+// uplink selection's emission does on the fly when the messages are produced on this GPU.
+// Also resets the union's state for the step.
+__global__ void __launch_bounds__(256)
+agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, RowState* uni, Ctrl* ctrl, u32 d) {
+    u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e == 0) {
+        uni->lo = 0; uni->cand_count = 0; uni->max_key = 0; uni->out_count = 0; uni->flags = 0;
+        uni->sum_sq = 0.0; uni->sel_sq = 0.0; uni->nnz = 0;
+    }
+    if (e >= total) return;
+    u32 j = up[e].x;
+    if (j >= d) { raise_status(ctrl, -5); next[e] = 0; return; }
+    next[e] = atomicExch(&head[j], e + 1);
+}
+
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
                   u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,

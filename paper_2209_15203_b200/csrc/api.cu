@@ -502,27 +502,13 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
     return TK_OK;
 }
 
-int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
-    if (!c || !aligned4(w_dev) || !aligned4(grads_dev) || !isfinite(alpha)) return TK_ERR_INVALID;
-    if (mode < 0 || mode > (TK_MODE_BIDIR | TK_MODE_EF)) return TK_ERR_INVALID;
+namespace {
+
+// Stages 2-4 on the messages in c->up.out (already threaded onto their chains).
+int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     const bool bidir = (mode & TK_MODE_BIDIR) != 0, with_ef = (mode & TK_MODE_EF) != 0;
-    if (with_ef && (!c->eps || c->K_down > c->ef_kdown)) return TK_ERR_INVALID;
-    cudaStream_t s = c->stream;
-    cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
-        e0 = c->ev[2 * c->ev_used];
-        e1 = c->ev[2 * c->ev_used + 1];
-        c->ev_used += 1;
-    }
-    // the first kernel of the selection also resets the state of the union / downlink selection
-    // ... and its last kernel threads every uplink entry onto its coordinate's chain (and, with
-    // error memories, zeroes the sent entries in eps)
     const bool diag = c->diagnostics != 0;
-    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0};
-    EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
-    int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
-                        &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
-    if (rc != TK_OK) return rc;
+    cudaStream_t s = c->stream;
     // with memories the step size is already inside the messages
     const float scale = with_ef ? 1.0f : alpha;
     u32 total = (u32)(c->N * c->K_up);
@@ -532,6 +518,7 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
                                              c->ctrl, (u32)c->d, diag ? 1 : 0);
     TK_LAUNCH_CHECK();
     c->launches += 1;
+    int rc = TK_OK;
     if (bidir && with_ef) {
         // Algorithm 2 with the server memory: delta now holds g = sum + delta everywhere; take
         // Top_K_down out of it (delta <- g - Top_K(g)) and apply it (w <- w - Top_K(g))
@@ -556,6 +543,72 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     c->last_mode = mode;
     c->last_kdown = c->K_down;
     return TK_OK;
+}
+
+bool step_args_ok(tk_ctx* c, float alpha, int mode) {
+    if (!c || !isfinite(alpha)) return false;
+    if (mode < 0 || mode > (TK_MODE_BIDIR | TK_MODE_EF)) return false;
+    if ((mode & TK_MODE_EF) && (!c->eps || c->K_down > c->ef_kdown)) return false;
+    return true;
+}
+
+}  // namespace
+
+int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
+    if (!step_args_ok(c, alpha, mode) || !aligned4(w_dev) || !aligned4(grads_dev)) return TK_ERR_INVALID;
+    const bool with_ef = (mode & TK_MODE_EF) != 0;
+    cudaStream_t s = c->stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
+        e0 = c->ev[2 * c->ev_used];
+        e1 = c->ev[2 * c->ev_used + 1];
+        c->ev_used += 1;
+    }
+    // the first kernel of the selection also resets the state of the union / downlink selection
+    // ... and its last kernel threads every uplink entry onto its coordinate's chain (and, with
+    // error memories, zeroes the sent entries in eps)
+    const bool diag = c->diagnostics != 0;
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0};
+    EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
+    int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
+                        &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
+    if (rc != TK_OK) return rc;
+    return run_server(c, w_dev, alpha, mode);
+}
+
+int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_t rows, float alpha, int mode) {
+    if (!step_args_ok(c, alpha, mode) || !aligned4(grads_local_dev)) return TK_ERR_INVALID;
+    if (row0 < 0 || rows < 1 || (int64_t)row0 + rows > c->N) return TK_ERR_INVALID;
+    const bool with_ef = (mode & TK_MODE_EF) != 0;
+    // this rank's slice of every per-row buffer
+    SelectBufs b = c->up;
+    b.rs += row0;
+    b.hist += (size_t)row0 * kHistBins;
+    b.smax += (size_t)row0 * kSampleSlots;
+    b.cand += (size_t)row0 * b.cap;
+    b.out += (size_t)row0 * (size_t)c->K_up;
+    float* eps = with_ef ? c->eps + (size_t)row0 * (size_t)c->d : nullptr;
+    LinkArgs link = {nullptr, nullptr, 0, 0, eps, (size_t)c->d, 0};  // chains are built after the exchange
+    EfArgs ef = {eps, alpha};
+    return run_select(c->stream, grads_local_dev, rows, c->d, c->K_up, b, c->ctrl, c->force_general != 0, nullptr,
+                      nullptr, &c->launches, nullptr, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0);
+}
+
+int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {
+    if (!c || !msgs_dev) return TK_ERR_INVALID;
+    *msgs_dev = c->up.out;
+    if (bytes_per_row) *bytes_per_row = (size_t)c->K_up * sizeof(uint2);
+    return TK_OK;
+}
+
+int tk_step_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
+    if (!step_args_ok(c, alpha, mode) || !aligned4(w_dev)) return TK_ERR_INVALID;
+    u32 total = (u32)(c->N * c->K_up);
+    agg_link_kernel<<<(total + 255) / 256, 256, 0, c->stream>>>(c->up.out, total, c->head, c->next, c->uni, c->ctrl,
+                                                                 (u32)c->d);
+    TK_LAUNCH_CHECK();
+    c->launches += 1;
+    return run_server(c, w_dev, alpha, mode);
 }
 
 int tk_step_host(tk_ctx* c, float* w_host, const float* grads_host, float alpha, int mode) {

@@ -7,7 +7,7 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2209_15203_b200 import replicas
+from paper_2209_15203_b200 import replicas, sharding
 
 
 def _free_port():
@@ -26,6 +26,14 @@ def _rank_main(rank, world, port, out):
         replicas.barrier()
         local_ms = 2.0 if rank == 0 else 5.0          # rank 1 is the slow replica
         value, ms = replicas.whole_job_throughput(local_ms, units_per_step=1000, steps=10)
+        # the uplink exchange of the sharded step: every rank fills its own rows of the message buffer
+        N, K = 6, 5
+        row0, rows = sharding.row_range(N, rank, world)
+        msgs = torch.full((N, K), -1, dtype=torch.int64)
+        msgs[row0:row0 + rows] = torch.arange(rows * K).view(rows, K) + 1000 * rank
+        sharding.all_gather_messages(msgs, row0, rows)
+        expect = torch.cat([torch.arange(rows * K).view(rows, K) + 1000 * r for r in range(world)])
+        assert torch.equal(msgs, expect), "rank %d does not hold all messages in worker order" % rank
         out.put((rank, replicas.world_size(), value, ms, replicas.max_over_ranks(float(rank))))
     finally:
         dist.destroy_process_group()
@@ -45,6 +53,13 @@ def test_two_replicas_report_the_slowest_rank():
     for rank, ws, value, ms, mx in results:
         assert ws == 2 and ms == 5.0 and mx == 1.0
         assert value == 2 * 1000 * 10 / 5e-3           # both replicas' units over the slowest time
+
+
+def test_row_ranges():
+    assert [sharding.row_range(8, r, 4) for r in range(4)] == [(0, 2), (2, 2), (4, 2), (6, 2)]
+    import pytest
+    with pytest.raises(ValueError):
+        sharding.row_range(7, 0, 2)
 
 
 def test_single_process_is_the_identity():
