@@ -166,6 +166,8 @@ def main():
                     "12 bytes per gradient value instead of 4")
     ap.add_argument("--sharded", action="store_true", help="with --gpus N > 1: shard the N workers over the ranks "
                     "(one all-gather of the messages per step) instead of running independent replicas")
+    ap.add_argument("--force-general", action="store_true", help="time the exact multi-pass path instead of the "
+                    "sampled single-pass one")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -203,6 +205,8 @@ def main():
     mode = binding.TK_MODE_BIDIR | (binding.TK_MODE_EF if args.ef else 0)
     if args.ef:
         ctx.tk_ef_attach()
+    if args.force_general:
+        ctx.tk_set_force_general(True)
 
     def barrier():
         replicas.barrier()

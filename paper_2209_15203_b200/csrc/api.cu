@@ -306,7 +306,7 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
-    const bool predict = !force_general && d >= 262144 && K * 64 <= d;
+    const bool predict = !force_general && d >= 131072 && K * 64 <= d;
     bool fused = ef.eps != nullptr && predict && ((((uintptr_t)x) ^ ((uintptr_t)ef.eps)) & 15u) == 0;
     if (ef.eps && !fused) {
         size_t n = (size_t)rows * (size_t)d;
