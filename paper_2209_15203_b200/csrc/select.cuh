@@ -818,14 +818,45 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             if (lane == 31) base = atomicAdd(&r->out_count, wtotal);
             base = __shfl_sync(0xffffffffu, base, 31);
         }
-        u32 slot = base + incl - mine;
+        const u32 slot0 = base + incl - mine;
+        // The entries of one thread go to different coordinates, so their memory round trips (the
+        // old value of w, the previous head of the chain) are independent: issue them all, then
+        // finish them all, instead of one dependent load-store pair after the other.
+        u32 fetched[kSelectRegs];
+        u32 slot = slot0;
+#pragma unroll
+        for (int k = 0; k < kSelectRegs; ++k) {
+            fetched[k] = 0;
+            if (eck[k] >= T) {
+                u32 idx = 0xffffffffu - (u32)eck[k];
+                if (slot < Keff && idx < 0x80000000u) {
+                    if (apply.w) fetched[k] = __float_as_uint(apply.w[idx]);
+                    if (link.head && idx < link.d)
+                        fetched[k] = atomicExch(&link.head[idx], (link.row_base + row) * (u32)out_stride + slot + 1);
+                }
+                ++slot;
+            }
+        }
+        slot = slot0;
 #pragma unroll
         for (int k = 0; k < kSelectRegs; ++k) {
             if (eck[k] >= T) {
                 u32 idx = 0xffffffffu - (u32)eck[k];
                 u32 bits = (u32)(eck[k] >> 32) | (((esign >> k) & 1u) << 31);
-                emit_entry(row, slot, Keff, idx, bits, orow, out_stride, apply, link, ctrl);
-                if (link.stats) sel_sq += (double)__uint_as_float(bits) * (double)__uint_as_float(bits);
+                if (slot >= Keff) {
+                    raise_status(ctrl, -5);
+                } else {
+                    orow[slot] = make_uint2(idx, bits);
+                    if (apply.w)
+                        apply.w[idx] = __fsub_rn(__uint_as_float(fetched[k]), __fmul_rn(apply.alpha, __uint_as_float(bits)));
+                    if (link.zero_src) link.zero_src[(size_t)row * link.zero_stride + idx] = 0.0f;
+                    if (link.head) {
+                        u32 e = (link.row_base + row) * (u32)out_stride + slot;
+                        if (idx < link.d) link.next[e] = fetched[k];
+                        else { link.next[e] = 0; raise_status(ctrl, -5); }
+                    }
+                    if (link.stats) sel_sq += (double)__uint_as_float(bits) * (double)__uint_as_float(bits);
+                }
                 ++slot;
             }
         }
