@@ -360,7 +360,11 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             u64 resident = (u64)di->sms * kFilterCtasPerSm;  // one wave: a second, partial wave runs at low occupancy
             u32 grid = (u32)(tiles < resident ? tiles : resident);
             u32 parts = 1;
-            if (tiles >= 4 * resident) parts = (u32)(nr < kFilterPartitions ? nr : kFilterPartitions);
+            if (tiles >= 4 * resident) {  // about one range per row, but never fewer than kFilterMinCpp CTAs per range
+                u32 most = grid / kFilterMinCpp;
+                parts = (u32)nr < most ? (u32)nr : most;
+                if (parts < 1) parts = 1;
+            }
             u32 cpp = grid / parts;
             size_t shm = (size_t)nr * sizeof(u64);
             if (fused && stats)
@@ -387,7 +391,11 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
                             (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl, (void*)&st};
             // without a prediction the multi-pass kernel is the streaming pass that gets timed
             if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
-            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(di->general_grid), dim3(kGeneralThreads), args,
+            // no more CTAs than tiles: a grid-wide barrier costs more the more CTAs take part
+            u64 gtiles = (u64)nr * b.tpr_general;
+            unsigned ggrid = (unsigned)(gtiles < (u64)di->general_grid ? gtiles : (u64)di->general_grid);
+            if (ggrid < 1) ggrid = 1;
+            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(ggrid), dim3(kGeneralThreads), args,
                                             0, stream) != cudaSuccess) {
                 cudaGetLastError();
                 return TK_ERR_CUDA;

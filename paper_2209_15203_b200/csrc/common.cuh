@@ -47,7 +47,12 @@ constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
 constexpr int kFilterEfUnroll = 3;     // with error memories a thread has two loads in flight per float4
 constexpr int kFilterEfTileVecs = kFilterThreads * kFilterEfUnroll;
-constexpr int kFilterPartitions = 8;   // the filter grid splits the tile space into this many ranges
+#ifndef TK_FILTER_MIN_CPP
+#define TK_FILTER_MIN_CPP 37
+#endif
+// The filter grid splits the tile space into ranges shared by at least this many CTAs each
+// (8 ranges on 296 CTAs; 37 ranges of 8 CTAs measured 3 % slower on the 32-row workload).
+constexpr int kFilterMinCpp = TK_FILTER_MIN_CPP;
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path

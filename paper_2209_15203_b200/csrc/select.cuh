@@ -747,7 +747,10 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                 u64 off = composite(key_of(e.y), e.x) - lo;
                 if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
-            if (kGrid) {
+            if (kGrid && CS == 1) {  // the whole list in one CTA: its own histogram is the total
+                __syncthreads();
+                for (int b = threadIdx.x; b < nb; b += kSelectThreads) sh_tot[b] = hist[b];
+            } else if (kGrid) {
                 u32* gh = ghist + (u32)(level % 3) * kHistBins;
                 __syncthreads();
                 for (int b = threadIdx.x; b < nb; b += kSelectThreads)
@@ -788,7 +791,9 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             T = lo;
             if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
         }
-        if (kGrid) {
+        if (kGrid && CS == 1) {
+            // nothing was exchanged
+        } else if (kGrid) {
             // leave ghist all zero for the next launch: once everybody has read the last level
             grid.sync();
             if (rank == 0)
