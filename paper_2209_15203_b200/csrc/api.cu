@@ -325,7 +325,10 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         // sample ~128*d/K values per row (about 128 members of the top K; fewer when that would take
         // more than kPredictMaxTurns loads per thread), as whole 128-byte lines
         const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
-        const int64_t max_turns = fused ? kPredictMaxTurns / 2 : kPredictMaxTurns;
+        int64_t max_turns = fused ? kPredictMaxTurns / 2 : kPredictMaxTurns;
+        // many rows: the sampling CTAs of all rows should fit few waves, so cap the loads per thread
+        // at what the two-CTAs-per-SM variant holds (the sample only sets how many candidates pass)
+        if (rows * kPredictCtas > 2 * (int64_t)di->sms) max_turns = fused ? kPredictLightTurns / 2 : kPredictLightTurns;
         int64_t want = (128 * (d / K) + per_turn - 1) / per_turn;
         int64_t lim = d / (8 * per_turn) < max_turns ? d / (8 * per_turn) : max_turns;
         turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
@@ -347,12 +350,16 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         EfArgs efb = {fused ? ef.eps + (size_t)r0 * (size_t)d : nullptr, ef.alpha};
         if (predict) {
             RowState* ar = r0 == 0 ? also_reset : nullptr;
-            if (fused)
-                predict_kernel<true><<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank,
-                                                                                             rs, smax, ar, efb);
+            const bool light = turns <= (fused ? kPredictLightTurns / 2 : kPredictLightTurns);
+            dim3 pg(kPredictCtas, nr);
+            if (fused && light)
+                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+            else if (fused)
+                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+            else if (light)
+                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
             else
-                predict_kernel<false><<<dim3(kPredictCtas, nr), kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank,
-                                                                                              rs, smax, ar, efb);
+                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             u32 tprf = fused ? b.tpr_filter_ef : b.tpr_filter;

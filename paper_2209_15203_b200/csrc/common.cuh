@@ -26,6 +26,7 @@ constexpr int kPredictCtas = 8;        // sampling CTAs per row
 constexpr int kPredictThreads = 1024;
 constexpr int kSampleSlots = kPredictCtas * kPredictThreads / 2;  // per-row sample maxima (one per thread pair)
 constexpr int kPredictMaxTurns = 10;   // 16-byte loads one sampling thread issues, all at once
+constexpr int kPredictLightTurns = 2;  // ... in the variant for many rows
 // Streaming passes.  Measured on B200: read bandwidth peaks with about 900-1150 threads and
 // 65-80 KB of loads in flight per SM and falls off sharply on either side (more resident
 // threads or deeper unrolling lose 20 %), so the filter kernel runs 2 CTAs of 448 threads

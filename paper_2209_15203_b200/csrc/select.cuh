@@ -51,8 +51,10 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->nnz = 0;
 }
 
-template <bool kEF>
-__global__ void __launch_bounds__(kPredictThreads)
+// kLight: at most kPredictLightTurns loads per thread; needs half the registers, so two CTAs
+// fit an SM (used when the rows are many and the sample per row is small).
+template <bool kEF, bool kLight>
+__global__ void __launch_bounds__(kPredictThreads, kLight ? 2 : 1)
 predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank,
                RowState* rs, u32* smax, RowState* also_reset, EfArgs ef) {
     __shared__ u32 sh_hist[kHistBins];
@@ -67,7 +69,9 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     // runs start at multiples of 32 elements
     const bool vec_ok = (((uintptr_t)xr) & 15u) == 0 && (!kEF || (((uintptr_t)er) & 15u) == 0);
     constexpr u32 kLinesPerTurn = 2 * kSampleSlots / 8;
-    constexpr int kTurns = kEF ? kPredictMaxTurns / 2 : kPredictMaxTurns;  // two loads per turn with memories
+    // two loads per turn with memories
+    constexpr int kTurns = kLight ? (kEF ? kPredictLightTurns / 2 : kPredictLightTurns)
+                                  : (kEF ? kPredictMaxTurns / 2 : kPredictMaxTurns);
     uint4 v[kTurns], m[kEF ? kTurns : 1];
 #pragma unroll
     for (int k = 0; k < kTurns; ++k) {
