@@ -33,7 +33,7 @@ UNIT = "elements/s"
 NOMINAL_HBM_BPS = 8e12
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch, from the ncu capture
-# summarised in profiles/filter_kernel_config5_rows2.md: (992.085 + 3.72) MB for 2 of the 8 workers,
+# summarised under profiles/ (filter kernel, 2 of the 8 workers): (992.085 + 3.72) MB,
 # scaled by the rows of the launch (None for any other workload, or once the kernel has changed)
 FILTER_TRAFFIC_PER_ROW_CONFIG5 = (992.085e6 + 3.72e6) / 2
 
