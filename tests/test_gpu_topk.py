@@ -50,6 +50,19 @@ def test_special_values():
     run_both((((-1.0) ** j) * (j + 1)).astype(np.float32), 33)  # closed form: the last K indices
 
 
+def test_nan_and_inf_are_ordered_by_bit_pattern():
+    # inputs are meant to be finite; if they are not, NaN (largest keys) and Inf are still selected
+    # exactly as the integer-key order says, on the sampled path and on the multi-pass path
+    rng = np.random.default_rng(8)
+    for d, K in ((300_000, 200), (20_000, 50)):
+        x = rng.standard_normal((2, d)).astype(np.float32)
+        x[0, [5, 77_77, d - 1]] = np.nan
+        x[0, 123] = -np.inf
+        x[1, 4_000] = np.float32(np.nan)
+        x[1, 4_001] = np.inf
+        run_both(x, K)
+
+
 def test_k_equals_d_and_k_one():
     rng = np.random.default_rng(1)
     x = rng.standard_normal((2, 30_001)).astype(np.float32)
