@@ -234,11 +234,12 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
     return L;
 }
 
-// CTAs per row of the cluster select: enough that a row's expected candidates sit in registers
-// (kSelectRegs per thread), at least 4 when there are few rows (latency), but never so many
-// that the clusters of all rows stop fitting in one wave.
+// CTAs per row of the cluster select: the kernel issues a fixed string of instructions per
+// register-held candidate and level, so few candidates per thread (about 4) on many SMs beats
+// many per thread on few; at least 4 CTAs when there are few rows, but never so many that the
+// clusters of all rows stop fitting in one wave.
 int cluster_size_for(int64_t entries, int64_t rows, int sms) {
-    int64_t per_cta = (int64_t)kSelectThreads * kSelectRegs;
+    int64_t per_cta = (int64_t)kSelectThreads * kSelectPerThread;
     int64_t need = (entries + per_cta - 1) / per_cta;
     int cs_need = 1;
     while (cs_need < 8 && cs_need < need) cs_need *= 2;

@@ -55,6 +55,10 @@ constexpr int kFilterEfTileVecs = kFilterThreads * kFilterEfUnroll;
 // (8 ranges on 296 CTAs; 37 ranges of 8 CTAs measured 3 % slower on the 32-row workload).
 constexpr int kFilterMinCpp = TK_FILTER_MIN_CPP;
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
+#ifndef TK_SELECT_PER_THREAD
+#define TK_SELECT_PER_THREAD 8
+#endif
+constexpr int kSelectPerThread = TK_SELECT_PER_THREAD;  // candidates per thread the cluster size aims at
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path
 constexpr u32 kRowNoFilter = 2u;       // RowState.flags: no filter pass has read this row

@@ -712,14 +712,17 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     const u32 rest = first + kSelectRegs * stride;  // entries from here on are re-read every level
 
     // this thread's entries first + k*stride, k < kSelectRegs, stay in registers as composite
-    // keys (0 = absent; a real entry's composite key is never 0) plus one sign bit each
+    // keys (0 = absent; a real entry's composite key is never 0) plus one sign bit each.
+    // Only the first `nslots` register slots can hold anything (the same for all threads of
+    // the row): the unrolled loops below skip the others.
+    const u32 nslots = min((u32)kSelectRegs, (C + stride - 1) / stride);
     u64 eck[kSelectRegs];
     u32 esign = 0;
 #pragma unroll
     for (int k = 0; k < kSelectRegs; ++k) {
         u32 i = first + (u32)k * stride;
         eck[k] = 0;
-        if (i < C) {
+        if ((u32)k < nslots && i < C) {
             uint2 e = list[i];
             eck[k] = composite(key_of(e.y), e.x);
             esign |= (e.y >> 31) << k;
@@ -743,6 +746,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             __syncthreads();
 #pragma unroll
             for (int k = 0; k < kSelectRegs; ++k) {
+                if ((u32)k >= nslots) break;
                 u64 off = eck[k] - lo;              // wraps to a huge value when eck < lo
                 if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
@@ -812,7 +816,10 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     double sel_sq = 0.0;
     u32 mine = 0;
 #pragma unroll
-    for (int k = 0; k < kSelectRegs; ++k) mine += eck[k] >= T ? 1u : 0u;
+    for (int k = 0; k < kSelectRegs; ++k) {
+        if ((u32)k >= nslots) break;
+        mine += eck[k] >= T ? 1u : 0u;
+    }
     {
         u32 lane = lane_id();
         u32 incl = mine;
@@ -836,6 +843,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
 #pragma unroll
         for (int k = 0; k < kSelectRegs; ++k) {
             fetched[k] = 0;
+            if ((u32)k >= nslots) break;
             if (eck[k] >= T) {
                 u32 idx = 0xffffffffu - (u32)eck[k];
                 if (slot < Keff && idx < 0x80000000u) {
@@ -849,6 +857,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         slot = slot0;
 #pragma unroll
         for (int k = 0; k < kSelectRegs; ++k) {
+            if ((u32)k >= nslots) break;
             if (eck[k] >= T) {
                 u32 idx = 0xffffffffu - (u32)eck[k];
                 u32 bits = (u32)(eck[k] >> 32) | (((esign >> k) & 1u) << 31);
