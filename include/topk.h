@@ -67,8 +67,9 @@ enum {
 /* Counters of the last step / selection, filled by tk_status(). */
 typedef struct tk_stats {
     int32_t device_status;    /* sticky TK_ERR_* raised by a kernel, 0 if none */
-    int32_t rows_general;     /* rows whose predicted threshold failed verification in the
-                                 last selection and were redone by the exact multi-pass path */
+    int32_t rows_general;     /* rows the exact multi-pass path handled in the last selection: rows whose
+                                 predicted threshold failed verification, or all rows when none was
+                                 predicted (short rows, K > d/64, tk_set_force_general) */
     int64_t union_size;       /* |U|: distinct indices in the last aggregate (<= N*K_up);
                                  |U|/d is the non-zero fraction of Section 4.2 */
     int64_t downlink_count;   /* entries applied to w in the last step */
@@ -87,7 +88,7 @@ size_t tk_workspace_bytes(int64_t d, int32_t N, int64_t K_up, int64_t K_down);
  * Eq. 1: minimise sum_q p_q F^q(w), w in R^d).
  *   out             receives the context
  *   d               1 <= d < 2^31
- *   N               >= 1
+ *   N               1 <= N <= 65535, with N * K_up < 2^31
  *   K_up, K_down    1 <= K <= d   (Section 4.2's K_uplink, K_downlink)
  *   p_host          [N] weights p_q, finite and >= 0 (copied; the sum is not checked)
  *   workspace_dev   device buffer of at least tk_workspace_bytes() bytes, 256-byte
