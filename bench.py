@@ -168,6 +168,10 @@ def main():
                     "(one all-gather of the messages per step) instead of running independent replicas")
     ap.add_argument("--force-general", action="store_true", help="time the exact multi-pass path instead of the "
                     "sampled single-pass one")
+    ap.add_argument("--no-graph", action="store_true", help="issue every step as plain stream launches instead of "
+                    "replaying captured CUDA graphs (tk_set_graph)")
+    ap.add_argument("--profile-every", type=int, default=4, help="timestamp the streaming kernel of every n-th timed "
+                    "step (such a step is issued as plain launches)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -196,7 +200,11 @@ def main():
     wl = W.workload(args.config, d=args.d or None, N=args.rows or None)
     K_down = wl.K_down[0]
     p = W.make_p(wl)
-    ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p)
+    # graphs need a capturable (non-default) stream; everything below runs on it
+    args.graph = not args.no_graph
+    run_stream = torch.cuda.Stream(dev) if args.graph else torch.cuda.current_stream(dev)
+    torch.cuda.set_stream(run_stream)
+    ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p, stream=run_stream)
     scale = W.scale_vector(wl, dev)
     nbuf = max(1, min(args.steps, 8))
     bufs = [W.make_grads(wl, s, dev, scale=scale) for s in range(nbuf)]
@@ -224,10 +232,14 @@ def main():
         def step(g):
             ctx.tk_step(w, g, wl.alpha, mode)
 
+    if args.graph:
+        ctx.tk_set_graph(True)
+        for s in range(nbuf):                 # capture every buffer's step before anything is timed
+            step(bufs[s % nbuf])
     for s in range(warmup):
         step(bufs[s % nbuf])
     st = ctx.tk_status()
-    ctx.tk_set_profile(True)
+    ctx.tk_set_profile(max(1, args.profile_every))
 
     sampler = ClockSampler(physical_gpu_index(local))
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -244,7 +256,7 @@ def main():
     launches = ctx.tk_launch_count() - launches0
     st = ctx.tk_status()
     sampler.join(timeout=2.0)
-    ctx.tk_set_profile(False)
+    ctx.tk_set_profile(0)
 
     elems = wl.N * wl.d
     value, ms_max = replicas.whole_job_throughput(ms, elems, args.steps, dev)
@@ -308,6 +320,8 @@ def main():
         cfg = W.describe(wl)
         cfg.update({"mode": "bidirectional with error memories" if args.ef else "bidirectional", "cold_inputs": "each step reads a %d MB gradient tensor (>> L2), "
                     "%d distinct tensors cycled" % (4 * elems // 10 ** 6, nbuf),
+                    "launch": ("CUDA graph replay; every %d-th step plain launches with timestamps around the "
+                               "streaming kernel" % max(1, args.profile_every)) if args.graph else "stream launches",
                     "parallelism": ("workers sharded over %d ranks, one all-gather per step" if args.sharded
                                     else "replicas x%d") % world})
         out = {

@@ -77,7 +77,7 @@ typedef struct tk_stats {
     int64_t cand_max;
     float   select_ms_sum;    /* device time of the streaming selection passes recorded since the
                                  previous tk_status call, and how many were recorded (both 0 */
-    int32_t select_samples;   /* unless tk_set_profile(ctx, 1); at most 256 are kept) */
+    int32_t select_samples;   /* unless tk_set_profile is on; at most 256 are kept) */
 } tk_stats;
 
 /* Bytes of device workspace tk_init needs for these sizes (0 if they are invalid). */
@@ -259,8 +259,21 @@ typedef struct tk_diag {
 int tk_set_diagnostics(tk_ctx* ctx, int on);
 int tk_diagnostics(tk_ctx* ctx, tk_diag* out, double* one_minus_gamma_up_host);
 
-/* Record device timestamps around the streaming selection pass of each step (0/1). */
-int tk_set_profile(tk_ctx* ctx, int on);
+/* Record device timestamps around the streaming selection pass of every `every`-th tk_step
+ * (0 = off, 1 = every step); tk_status reports their sum.  A timestamped step is always issued
+ * as plain launches, also when tk_set_graph is on. */
+int tk_set_profile(tk_ctx* ctx, int every);
+
+/*
+ * Replay steps as CUDA graphs (0/1, off by default).  A step is six to ten small dependent
+ * launches around one long one; for small workloads the launch gaps are a tenth of the step.
+ * With this on, the first tk_step with a given (w_dev, grads_dev, alpha, mode, K_down) captures
+ * the launches into a graph and every later call with the same arguments replays it (up to 16
+ * distinct argument sets are kept, least recently used dropped).  Needs a context created on a
+ * non-default stream; bypassed for the steps tk_set_profile timestamps and while the caller is
+ * itself capturing the stream.  Results are identical.
+ */
+int tk_set_graph(tk_ctx* ctx, int on);
 
 /*
  * Testing aid: force every selection of this context down the exact multi-pass

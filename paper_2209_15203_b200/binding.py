@@ -23,7 +23,7 @@ TK_MODE_EF = 2
 EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
            "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
-           "tk_set_force_general", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
+           "tk_set_force_general", "tk_set_graph", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
 
 class TkError(RuntimeError):
@@ -98,6 +98,8 @@ def load(build_if_missing: bool = True):
     lib.tk_status.argtypes = [vp, ctypes.POINTER(tk_stats)]
     lib.tk_set_profile.argtypes = [vp, ctypes.c_int]
     lib.tk_set_force_general.argtypes = [vp, ctypes.c_int]
+    lib.tk_set_graph.argtypes = [vp, ctypes.c_int]
+    lib.tk_set_graph.restype = ctypes.c_int
     lib.tk_launch_count.argtypes = [vp]
     lib.tk_launch_count.restype = i64
     lib.tk_destroy.argtypes = [vp]
@@ -263,8 +265,12 @@ class Context:
             _check(rc, "tk_status")
         return st
 
-    def tk_set_profile(self, on: bool) -> None:
-        _check(load().tk_set_profile(self._h, 1 if on else 0), "tk_set_profile")
+    def tk_set_profile(self, every: int) -> None:
+        """0 = off; n = timestamp the streaming pass of every n-th step."""
+        _check(load().tk_set_profile(self._h, int(every)), "tk_set_profile")
+
+    def tk_set_graph(self, on: bool) -> None:
+        _check(load().tk_set_graph(self._h, 1 if on else 0), "tk_set_graph")
 
     def tk_set_force_general(self, on: bool) -> None:
         _check(load().tk_set_force_general(self._h, 1 if on else 0), "tk_set_force_general")

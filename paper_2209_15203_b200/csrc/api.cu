@@ -186,7 +186,8 @@ struct tk_ctx {
     // host state
     int force_general = 0;
     int diagnostics = 0;
-    int profile = 0;
+    int profile = 0;           // 0 = off, n = timestamp the streaming pass of every n-th step
+    int64_t steps_seen = 0;
     int last_mode = -1;
     int64_t last_kdown = 0;
     int64_t launches = 0;
@@ -200,6 +201,21 @@ struct tk_ctx {
     float* delta = nullptr;    // [d]
     SelectBufs down;           // selection over the dense server vector (1 row of d)
     int64_t ef_kdown = 0;      // largest K_down the attached buffers serve
+    // captured steps (tk_set_graph)
+    struct StepKey {
+        float* w; const float* g; float alpha; int mode; int64_t K_down; int force_general, diagnostics;
+        float* eps;
+        bool operator==(const StepKey& o) const {
+            return w == o.w && g == o.g && memcmp(&alpha, &o.alpha, sizeof alpha) == 0 && mode == o.mode &&
+                   K_down == o.K_down && force_general == o.force_general && diagnostics == o.diagnostics && eps == o.eps;
+        }
+    };
+    struct StepGraph { StepKey key; cudaGraphExec_t exec; int64_t launches; uint64_t used; };
+    static constexpr int kMaxGraphs = 16;
+    StepGraph graphs[kMaxGraphs] = {};
+    int n_graphs = 0;
+    uint64_t graph_clock = 0;
+    int use_graphs = 0;
 };
 
 namespace {
@@ -570,12 +586,84 @@ bool step_args_ok(tk_ctx* c, float alpha, int mode) {
 
 }  // namespace
 
+namespace {
+int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode, bool timed);
+
+void drop_graphs(tk_ctx* c) {
+    for (int i = 0; i < c->n_graphs; ++i) cudaGraphExecDestroy(c->graphs[i].exec);
+    c->n_graphs = 0;
+}
+}  // namespace
+
 int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
     if (!step_args_ok(c, alpha, mode) || !aligned4(w_dev) || !aligned4(grads_dev)) return TK_ERR_INVALID;
+    // Replay a captured graph of this very step (same buffers, same settings) when asked to.
+    // Not for a step whose streaming pass is being timestamped, not on the legacy default stream (it
+    // cannot be captured), not when the caller is itself capturing this stream.
+    const bool timed = c->profile > 0 && (c->steps_seen++ % c->profile) == 0;
+    if (c->use_graphs && !timed && c->stream != nullptr) {
+        cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(c->stream, &st) == cudaSuccess && st == cudaStreamCaptureStatusNone) {
+            tk_ctx::StepKey key = {w_dev, grads_dev, alpha, mode, c->K_down, c->force_general, c->diagnostics,
+                                   (mode & TK_MODE_EF) ? c->eps : nullptr};
+            tk_ctx::StepGraph* hit = nullptr;
+            for (int i = 0; i < c->n_graphs; ++i)
+                if (c->graphs[i].key == key) hit = &c->graphs[i];
+            if (!hit) {
+                int64_t before = c->launches;
+                if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+                    cudaGetLastError();
+                    return TK_ERR_CUDA;
+                }
+                int rc = enqueue_step(c, w_dev, grads_dev, alpha, mode, false);
+                cudaGraph_t graph = nullptr;
+                cudaError_t ce = cudaStreamEndCapture(c->stream, &graph);
+                int64_t per_step = c->launches - before;
+                c->launches = before;
+                if (rc != TK_OK || ce != cudaSuccess || !graph) {
+                    if (graph) cudaGraphDestroy(graph);
+                    cudaGetLastError();
+                    return rc != TK_OK ? rc : TK_ERR_CUDA;
+                }
+                cudaGraphExec_t exec = nullptr;
+                ce = cudaGraphInstantiate(&exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (ce != cudaSuccess) {
+                    cudaGetLastError();
+                    return TK_ERR_CUDA;
+                }
+                int slot = c->n_graphs;
+                if (slot == tk_ctx::kMaxGraphs) {  // evict the least recently used
+                    slot = 0;
+                    for (int i = 1; i < c->n_graphs; ++i)
+                        if (c->graphs[i].used < c->graphs[slot].used) slot = i;
+                    cudaGraphExecDestroy(c->graphs[slot].exec);
+                } else {
+                    c->n_graphs += 1;
+                }
+                c->graphs[slot] = tk_ctx::StepGraph{key, exec, per_step, 0};
+                hit = &c->graphs[slot];
+            }
+            hit->used = ++c->graph_clock;
+            if (cudaGraphLaunch(hit->exec, c->stream) != cudaSuccess) {
+                cudaGetLastError();
+                return TK_ERR_CUDA;
+            }
+            c->launches += hit->launches;
+            c->last_mode = mode;
+            c->last_kdown = c->K_down;
+            return TK_OK;
+        }
+    }
+    return enqueue_step(c, w_dev, grads_dev, alpha, mode, timed);
+}
+
+namespace {
+int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode, bool timed) {
     const bool with_ef = (mode & TK_MODE_EF) != 0;
     cudaStream_t s = c->stream;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (c->profile && c->ev_ready && c->ev_used < kMaxEvents) {
+    if (timed && c->ev_ready && c->ev_used < kMaxEvents) {
         e0 = c->ev[2 * c->ev_used];
         e1 = c->ev[2 * c->ev_used + 1];
         c->ev_used += 1;
@@ -591,6 +679,7 @@ int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mo
     if (rc != TK_OK) return rc;
     return run_server(c, w_dev, alpha, mode);
 }
+}  // namespace
 
 int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_t rows, float alpha, int mode) {
     if (!step_args_ok(c, alpha, mode) || !aligned4(grads_local_dev)) return TK_ERR_INVALID;
@@ -699,6 +788,7 @@ int tk_ef_attach(tk_ctx* c, void* mem_dev, size_t bytes) {
         cudaGetLastError();
         return TK_ERR_CUDA;
     }
+    drop_graphs(c);  // captured steps hold the old memories' addresses
     c->eps = (float*)base;
     c->delta = (float*)(base + off_delta);
     c->down = down;
@@ -865,7 +955,8 @@ int tk_set_profile(tk_ctx* c, int on) {
             if (cudaEventCreate(&c->ev[i]) != cudaSuccess) return TK_ERR_CUDA;
         c->ev_ready = true;
     }
-    c->profile = on ? 1 : 0;
+    c->profile = on > 0 ? on : 0;
+    c->steps_seen = 0;
     c->ev_used = 0;
     return TK_OK;
 }
@@ -917,6 +1008,13 @@ int tk_diagnostics(tk_ctx* c, tk_diag* out, double* one_minus_gamma_up_host) {
     return TK_OK;
 }
 
+int tk_set_graph(tk_ctx* c, int on) {
+    if (!c) return TK_ERR_INVALID;
+    c->use_graphs = on ? 1 : 0;
+    if (!on) drop_graphs(c);
+    return TK_OK;
+}
+
 int tk_set_force_general(tk_ctx* c, int on) {
     if (!c) return TK_ERR_INVALID;
     c->force_general = on ? 1 : 0;
@@ -927,6 +1025,7 @@ int64_t tk_launch_count(tk_ctx* c) { return c ? c->launches : 0; }
 
 void tk_destroy(tk_ctx* c) {
     if (!c) return;
+    drop_graphs(c);
     if (c->ev_ready)
         for (int i = 0; i < 2 * kMaxEvents; ++i) cudaEventDestroy(c->ev[i]);
     if (c->stage_g) cudaFree(c->stage_g);

@@ -209,6 +209,39 @@ def test_diagnostics_match_the_oracle():
         ctx.close()
 
 
+def test_graph_replay_matches_direct_launches():
+    wl = W.workload(2, d=500_000, N=4)
+    p = W.make_p(wl)
+    bufs = [W.make_grads(wl, s, DEV) for s in range(3)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for ef in (False, True):
+        mode = 1 | (binding.TK_MODE_EF if ef else 0)
+        direct = binding.Context(wl.d, wl.N, wl.K_up, wl.K_up, p)
+        with torch.cuda.stream(side):
+            graphed = binding.Context(wl.d, wl.N, wl.K_up, wl.K_up, p, stream=side)
+            graphed.tk_set_graph(True)
+        if ef:
+            direct.tk_ef_attach()
+            graphed.tk_ef_attach()
+        wa, wb = W.make_w(wl, DEV), W.make_w(wl, DEV)
+        torch.cuda.synchronize()
+        for s in range(9):                       # every buffer is captured once and replayed twice
+            kd = wl.K_up if s < 6 else 7         # a new K_down is a new graph
+            direct.tk_set_kdown(kd)
+            graphed.tk_set_kdown(kd)
+            direct.tk_step(wa, bufs[s % 3], wl.alpha, mode)
+            with torch.cuda.stream(side):
+                graphed.tk_step(wb, bufs[s % 3], wl.alpha, mode)
+        torch.cuda.synchronize()
+        assert graphed.tk_status().device_status == 0
+        assert torch.equal(wa.view(torch.int32), wb.view(torch.int32))
+        assert graphed.tk_launch_count() == direct.tk_launch_count()
+        ia, va = direct.tk_last_downlink()
+        ib, vb = graphed.tk_last_downlink()
+        assert torch.equal(ia, ib) and torch.equal(va.view(torch.int32), vb.view(torch.int32))
+
+
 def test_bad_arguments_are_rejected():
     wl = W.workload(1, d=1000)
     ctx = make_ctx(wl, 10)
