@@ -39,6 +39,7 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
                   u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
                   int stats) {
+    dependency_wait();   // the chains are built by the kernel before
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
     u32 j = 0;

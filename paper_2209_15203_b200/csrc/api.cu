@@ -266,6 +266,43 @@ int cluster_size_for(int64_t entries, int64_t rows, int sms) {
     return cs < cs_fill ? cs : cs_fill;
 }
 
+#ifndef TK_PDL
+#define TK_PDL 1
+#endif
+
+// Launch with the programmatic-serialization attribute (the kernel calls dependency_wait()) and,
+// optionally, a cluster size.
+template <typename... KArgs, typename... Args>
+int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster,
+                     Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (cluster > 0) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (TK_PDL) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n;
+    if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return TK_OK;
+}
+
 #define TK_LAUNCH_CHECK()                                   \
     do {                                                    \
         if (cudaGetLastError() != cudaSuccess) return TK_ERR_CUDA; \
@@ -273,26 +310,9 @@ int cluster_size_for(int64_t entries, int64_t rows, int sms) {
 
 int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, size_t list_stride, u32 cap,
                   RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(rows * cs), 1, 1);
-    cfg.blockDim = dim3(kSelectThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cs;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     u32* no_ghist = nullptr;
-    if (cudaLaunchKernelEx(&cfg, select_kernel<false>, lists, list_stride, cap, rs, K, out, out_stride, apply, link, ctrl,
-                           no_ghist) !=
-        cudaSuccess) {
-        cudaGetLastError();
-        return TK_ERR_CUDA;
-    }
-    return TK_OK;
+    return launch_dependent(select_kernel<false>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, lists,
+                            list_stride, cap, rs, K, out, out_stride, apply, link, ctrl, no_ghist);
 }
 
 // One long list selected by the whole grid (cooperative launch).
@@ -392,14 +412,18 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             u32 cpp = grid / parts;
             size_t shm = (size_t)nr * sizeof(u64);
             if (fused && stats)
-                filter_kernel<true, true><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
+                rc = launch_dependent(filter_kernel<true, true>, dim3(grid), dim3(kFilterThreads), shm, stream, 0, xb, nr, d, tprf,
+                                      parts, cpp, rs, cand, b.cap, efb);
             else if (fused)
-                filter_kernel<true, false><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
+                rc = launch_dependent(filter_kernel<true, false>, dim3(grid), dim3(kFilterThreads), shm, stream, 0, xb, nr, d, tprf,
+                                      parts, cpp, rs, cand, b.cap, efb);
             else if (stats)
-                filter_kernel<false, true><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
+                rc = launch_dependent(filter_kernel<false, true>, dim3(grid), dim3(kFilterThreads), shm, stream, 0, xb, nr, d, tprf,
+                                      parts, cpp, rs, cand, b.cap, efb);
             else
-                filter_kernel<false, false><<<grid, kFilterThreads, shm, stream>>>(xb, nr, d, tprf, parts, cpp, rs, cand, b.cap, efb);
-            TK_LAUNCH_CHECK();
+                rc = launch_dependent(filter_kernel<false, false>, dim3(grid), dim3(kFilterThreads), shm, stream, 0, xb, nr, d, tprf,
+                                      parts, cpp, rs, cand, b.cap, efb);
+            if (rc != TK_OK) return rc;
             if (fused) xb = efb.eps;  // the compensated vector now sits in eps: what a re-filter must read
             if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 2;
@@ -545,12 +569,12 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     const float scale = with_ef ? 1.0f : alpha;
     u32 total = (u32)(c->N * c->K_up);
     u32 blocks = (total + 255) / 256;
-    agg_reduce_kernel<<<blocks, 256, 0, s>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->uni, c->U,
-                                             c->ucap, w_dev, scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : nullptr,
-                                             c->ctrl, (u32)c->d, diag ? 1 : 0);
-    TK_LAUNCH_CHECK();
+    int rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(256), 0, s, 0, (const uint2*)c->up.out, total,
+                              (u32)c->K_up, (const float*)c->p, c->head, (const u32*)c->next, c->uni, c->U, c->ucap, w_dev,
+                              scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : (float*)nullptr, c->ctrl, (u32)c->d,
+                              diag ? 1 : 0);
+    if (rc != TK_OK) return rc;
     c->launches += 1;
-    int rc = TK_OK;
     if (bidir && with_ef) {
         // Algorithm 2 with the server memory: delta now holds g = sum + delta everywhere; take
         // Top_K_down out of it (delta <- g - Top_K(g)) and apply it (w <- w - Top_K(g))

@@ -130,6 +130,15 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 
 __device__ __forceinline__ u32 lane_id() { return threadIdx.x & 31; }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization
+// attribute may become resident while its predecessor in the stream still runs; it must call
+// dependency_wait() before it touches anything the predecessor produces (the call returns at
+// once when the kernel was launched the ordinary way).  A predecessor calls
+// allow_dependents() as early as it likes: the dependent's launch latency then overlaps the
+// predecessor's run instead of following it.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // *dst += sum over the warp of v, accumulated in double.  All lanes call.
 __device__ __forceinline__ void warp_add_double(double* dst, double v) {
 #pragma unroll

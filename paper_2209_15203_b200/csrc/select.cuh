@@ -61,6 +61,7 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
     __shared__ u32 sh_ticket;
+    allow_dependents();  // the filter kernel may take its place on the SMs; it waits for this grid to end
     const int row = blockIdx.y;
     const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;   // 0 .. 2*kSampleSlots-1
     if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
@@ -376,6 +377,7 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
     __shared__ u32 sh_n[kFilterThreads / 32];
     const u32 part = blockIdx.x / cpp;
     if (part >= parts) return;
+    dependency_wait();  // the bounds come from the sampling kernel
     for (int r = threadIdx.x; r < rows; r += kFilterThreads) sh_lo[r] = rs[r].lo;
     if (threadIdx.x < kFilterThreads / 32) sh_n[threadIdx.x] = 0;
     __syncthreads();
@@ -496,6 +498,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
     __shared__ uint2 sh_buf[(kGeneralThreads / 32) * kStageSlots];
     __shared__ u32 sh_n[kGeneralThreads / 32];
     cg::grid_group grid = cg::this_grid();
+    allow_dependents();  // the uplink select may queue up behind this grid
 
     // Which rows failed verification?  Nothing below modifies a RowState before
     // the first grid-wide barrier, so every CTA sees the same answer.
@@ -700,6 +703,8 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     __shared__ u32 sh_res[2];
     cg::cluster_group cluster = cg::this_cluster();
     cg::grid_group grid = cg::this_grid();
+    dependency_wait();   // candidates and bounds come from the kernels before
+    allow_dependents();
     const u32 CS = kGrid ? gridDim.x : cluster.num_blocks();
     const u32 rank = kGrid ? blockIdx.x : cluster.block_rank();
     const u32 row = kGrid ? 0u : blockIdx.x / CS;
