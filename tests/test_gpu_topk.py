@@ -101,6 +101,14 @@ def test_predicted_path_large_rows():
     run_both(G.cpu().numpy(), wl.K_up, x_dev=G)
 
 
+@pytest.mark.parametrize("K", [15_000, 40_000, 300_000])
+def test_large_k_on_long_rows(K):
+    # 1 % (sampled path), 2.7 % and 20 % (beyond d/64: multi-pass path with large candidate lists)
+    wl = W.workload(3, d=1_500_000, N=3)
+    G = W.make_grads(wl, 2, DEV)
+    run_both(G.cpu().numpy(), K, x_dev=G)
+
+
 def test_rows_whose_prediction_must_fail():
     d, K = 1_200_000, 1_000
     rng = np.random.default_rng(4)
