@@ -46,7 +46,10 @@ constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads
 constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
 constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
-constexpr int kFilterEfUnroll = 3;     // with error memories a thread has two loads in flight per float4
+#ifndef TK_FILTER_EF_UNROLL
+#define TK_FILTER_EF_UNROLL 2
+#endif
+constexpr int kFilterEfUnroll = TK_FILTER_EF_UNROLL;  // with error memories a thread has two loads in flight per float4
 constexpr int kFilterEfTileVecs = kFilterThreads * kFilterEfUnroll;
 #ifndef TK_FILTER_MIN_CPP
 #define TK_FILTER_MIN_CPP 37
