@@ -22,13 +22,14 @@ _lib = None
 # Contraction must stay off so that p*v and alpha*s are rounded before the
 # add/subtract (two roundings per term), and no fast-math reassociation.
 _CFLAGS = ["-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC", "-pthread"]
+_LDLIBS = ["-lm"]
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle if the shared object is missing or older than its source."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.run(["gcc", *_CFLAGS, "-o", tmp, _SRC], check=True)
+        subprocess.run(["gcc", *_CFLAGS, "-o", tmp, _SRC, *_LDLIBS], check=True)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -48,6 +49,8 @@ def _load():
         lib.ref_step.argtypes = [f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
                                  i32p, f32p, f32p, u8p, i32p, f32p, ctypes.c_void_p, ctypes.c_int]
         lib.ref_step.restype = ctypes.c_int
+        lib.ref_rho.argtypes = [f32p, f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int, ctypes.c_int]
+        lib.ref_rho.restype = ctypes.c_double
         lib.ref_lost_energy.argtypes = [f32p, i64, i32p, i64]
         lib.ref_lost_energy.restype = ctypes.c_double
         lib.ref_step_ef.argtypes = [f32p, f32p, f32p, f32p, i64, i64, i64, i64, f32p, ctypes.c_float, ctypes.c_int,
@@ -196,3 +199,19 @@ def ref_lost_energy(x, idx) -> float:
     x = _f32(x).reshape(-1)
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     return float(_load().ref_lost_energy(_ptr(x), x.size, _ptr(idx), idx.size))
+
+
+def ref_rho(G, eps, delta, K_up: int, K_down: int, p, alpha: float, mode: int,
+            nthreads: Optional[int] = None) -> float:
+    """The gap constant of one iteration: rho_hat (mode 0) or rho (mode 1).  eps / delta are the
+    memories before the iteration; None = memory-free (then the step size cancels)."""
+    G = _f32(G)
+    p = _f32(p)
+    N, d = G.shape
+    eps = None if eps is None else _f32(eps)
+    delta = None if delta is None else _f32(delta)
+    nt = default_threads() if nthreads is None else nthreads
+    r = _load().ref_rho(_ptr(G), _ptr(eps), _ptr(delta), N, d, K_up, K_down, _ptr(p), ctypes.c_float(alpha), mode, nt)
+    if r < 0:
+        raise ValueError("ref_rho rejected its arguments")
+    return float(r)

@@ -44,6 +44,7 @@
 #include <stdlib.h>
 #include <string.h>
 #include <pthread.h>
+#include <math.h>
 
 typedef struct {
     uint32_t key; /* magnitude key */
@@ -358,4 +359,98 @@ double ref_lost_energy(const float *x, int64_t d, const int32_t *idx, int64_t K)
     }
     free(sent);
     return total > 0.0 ? lost / total : 0.0;
+}
+
+/*
+ * The gap constants of the convergence analysis, as the experiments estimate them per
+ * iteration (Section 4, "Convergence Bound Constants"; Assumptions on the gap, uni- and
+ * bidirectional).  With  a^q = eps^q + alpha g^q  (or a^q = g^q and delta = 0 for the
+ * memory-free iteration, where the step size cancels from the ratio), D_a = sum_q p_q a^q,
+ * D_g = sum_q p_q g^q and S = sum_q p_q Top_{K_up}(a^q):
+ *   mode 0:  rho_hat = || Top_K(D_a) - S ||_2                                / || scale D_g ||_2
+ *   mode 1:  rho     = || Top_K(delta + D_a) - Top_K(delta + S) ||_2         / || scale D_g ||_2
+ * with K = K_down for the server-side Top_K, scale = alpha with memories and 1 without.
+ * (The assumptions write Top_K(p_q a) where the algorithms write p_q Top_K(a); they agree for
+ * p_q > 0 and the algorithms' form is used.)  The dense sums are formed like everything else
+ * here: fp32, worker order, one rounding per multiply and per add; the norms in double.
+ * eps and delta are the memories BEFORE the iteration (NULL = zero / memory-free).
+ * Returns the ratio, 0 when the denominator is 0, or -1 on bad arguments.
+ */
+double ref_rho(const float *G, const float *eps, const float *delta, int64_t N, int64_t d,
+               int64_t K_up, int64_t K_down, const float *p, float alpha, int mode, int nthreads)
+{
+    if (!G || !p || N < 1 || d < 1 || K_up < 1 || K_up > d || K_down < 1 || K_down > d || (mode != 0 && mode != 1))
+        return -1.0;
+    double result = -1.0;
+    const int memories = eps != NULL;
+    float *a = (float *)malloc((size_t)(N * d) * sizeof *a);
+    float *Da = (float *)malloc((size_t)d * sizeof *Da);
+    float *Dg = (float *)malloc((size_t)d * sizeof *Dg);
+    float *S = (float *)malloc((size_t)d * sizeof *S);
+    float *left = (float *)calloc((size_t)d, sizeof *left);
+    float *right = (float *)calloc((size_t)d, sizeof *right);
+    uint8_t *touched = (uint8_t *)malloc((size_t)d);
+    int32_t *up_idx = (int32_t *)malloc((size_t)(N * K_up) * sizeof *up_idx);
+    float *up_val = (float *)malloc((size_t)(N * K_up) * sizeof *up_val);
+    int32_t *t_idx = (int32_t *)malloc((size_t)K_down * sizeof *t_idx);
+    float *t_val = (float *)malloc((size_t)K_down * sizeof *t_val);
+    if (!a || !Da || !Dg || !S || !left || !right || !touched || !up_idx || !up_val || !t_idx || !t_val) goto done;
+
+    for (int64_t q = 0; q < N; ++q)
+        for (int64_t j = 0; j < d; ++j) {
+            if (memories) {
+                volatile float scaled = alpha * G[q * d + j];
+                volatile float v = eps[q * d + j] + scaled;
+                a[q * d + j] = v;
+            } else {
+                a[q * d + j] = G[q * d + j];
+            }
+        }
+    for (int64_t j = 0; j < d; ++j) {
+        float sa = 0.0f, sg = 0.0f;
+        for (int64_t q = 0; q < N; ++q) {
+            volatile float ta = p[q] * a[q * d + j];
+            volatile float na = sa + ta;
+            sa = na;
+            volatile float tg = p[q] * G[q * d + j];
+            volatile float ng = sg + tg;
+            sg = ng;
+        }
+        Da[j] = sa;
+        Dg[j] = sg;
+    }
+    if (ref_topk_rows(a, N, d, K_up, up_idx, up_val, nthreads) != 0) goto done;
+    if (ref_aggregate(up_idx, up_val, N, K_up, p, d, S, touched) != 0) goto done;
+    if (mode == 1 && delta) {
+        for (int64_t j = 0; j < d; ++j) {
+            volatile float va = delta[j] + Da[j];
+            Da[j] = va;
+            volatile float vs = S[j] + delta[j];
+            S[j] = vs;
+        }
+    }
+    /* left = Top_K(D_a [+ delta]) */
+    if (ref_topk(Da, d, K_down, t_idx, t_val) != 0) goto done;
+    for (int64_t k = 0; k < K_down; ++k) left[t_idx[k]] = t_val[k];
+    /* right = S (mode 0) or Top_K(S [+ delta]) (mode 1) */
+    if (mode == 1) {
+        if (ref_topk(S, d, K_down, t_idx, t_val) != 0) goto done;
+        for (int64_t k = 0; k < K_down; ++k) right[t_idx[k]] = t_val[k];
+    } else {
+        memcpy(right, S, (size_t)d * sizeof *S);
+    }
+    {
+        double num = 0.0, den = 0.0;
+        for (int64_t j = 0; j < d; ++j) {
+            double df = (double)left[j] - (double)right[j];
+            num += df * df;
+            double g = (memories ? (double)alpha : 1.0) * (double)Dg[j];
+            den += g * g;
+        }
+        result = den > 0.0 ? sqrt(num) / sqrt(den) : 0.0;
+    }
+done:
+    free(a); free(Da); free(Dg); free(S); free(left); free(right); free(touched);
+    free(up_idx); free(up_val); free(t_idx); free(t_val);
+    return result;
 }

@@ -269,3 +269,34 @@ def test_lost_energy_closed_forms_and_bound():
     v = oracle.ref_lost_energy(r, idx)
     assert 0 < v <= (5000 - 50) / 5000
     assert abs(oracle.ref_lost_energy((r * np.float32(0.25)).astype(np.float32), idx) - v) < 1e-12
+
+
+def test_gap_constants_hand_example_and_special_cases():
+    g = _read_golden("alg2_first_iteration.txt")
+    G = np.array([g["g1"], g["g2"], g["g3"]], np.float32)
+    p = np.array(g["p"], np.float32)
+    den = g["rho_sq_den"][0]
+    assert abs(oracle.ref_rho(G, None, None, 2, 2, p, 0.5, 0) - (g["rho_hat_sq_num"][0] / den) ** 0.5) < 1e-12
+    assert abs(oracle.ref_rho(G, None, None, 2, 2, p, 0.5, 1) - (g["rho_sq_num"][0] / den) ** 0.5) < 1e-12
+    # one worker: the aggregate of its message IS Top_K of the sum, both constants vanish
+    rng = np.random.default_rng(31)
+    x = rng.standard_normal((1, 4000)).astype(np.float32)
+    one = np.ones(1, np.float32)
+    assert oracle.ref_rho(x, None, None, 40, 40, one, 1.0, 0) == 0.0
+    assert oracle.ref_rho(x, None, None, 40, 40, one, 1.0, 1) == 0.0
+    # no compression at all: nothing differs
+    y = rng.standard_normal((3, 50)).astype(np.float32)
+    w3 = np.array([0.5, 0.25, 0.25], np.float32)
+    assert oracle.ref_rho(y, None, None, 50, 50, w3, 1.0, 0) == 0.0
+    # with memories at zero and alpha a power of two the ratio equals the memory-free one
+    z = rng.standard_normal((4, 3000)).astype(np.float32)
+    w4 = np.full(4, 0.25, np.float32)
+    free = oracle.ref_rho(z, None, None, 30, 30, w4, 1.0, 1)
+    mem = oracle.ref_rho(z, np.zeros_like(z), np.zeros(3000, np.float32), 30, 30, w4, 0.25, 1)
+    assert free > 0 and abs(free - mem) < 1e-12
+    # the toy example's message: workers that disagree make the unidirectional gap large
+    c = np.array([1.0, 5.0, 10.0], np.float32)
+    wv = np.full(100, 5.4, np.float32)
+    wv[::7] += 0.3
+    Gq = (wv[None, :] - c[:, None]).astype(np.float32)
+    assert oracle.ref_rho(Gq, None, None, 1, 1, np.full(3, 1 / 3, np.float32), 0.01, 0) > 1.0
