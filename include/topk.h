@@ -240,10 +240,16 @@ int tk_last_downlink(tk_ctx* ctx, int32_t* idx_out_dev, float* val_out_dev, int6
 int tk_status(tk_ctx* ctx, tk_stats* out);
 
 /*
- * The paper's per-step diagnostics that do not need the uncompressed aggregate.
+ * The paper's per-step diagnostics.
  *   tk_set_diagnostics(ctx, 1)  makes the following steps also accumulate sums of squares
  *        (one fused multiply-add per value in the streaming pass, fp32 per thread, double across
- *        threads) and count the non-zeros of the aggregate.  Off by default.
+ *        threads) and count the non-zeros of the aggregate: cheap.
+ *   tk_set_diagnostics(ctx, 2)  adds the estimate of the gap constant of the convergence analysis
+ *        (rho_hat / rho, the paper's Table 1).  That needs what the method itself never forms,
+ *        the dense sum of the workers' vectors and its Top_K: the gradients are read a second
+ *        time and one more dense selection runs, so a step takes about twice as long.  The call
+ *        allocates 8*d bytes plus selection scratch with cudaMalloc (freed by tk_destroy).
+ *   tk_set_diagnostics(ctx, 0)  off (the default).
  *   tk_diagnostics              synchronises and reports, for the last step:
  */
 typedef struct tk_diag {
@@ -254,9 +260,15 @@ typedef struct tk_diag {
     double one_minus_gamma_up_max;  /* max_q ||Top_K(a^q) - a^q||^2 / ||a^q||^2: the "1 - gamma" estimate of the
                                        appendix for the uplink compressions (<= (d - K_up)/d by Eq. "topk_bound") */
     double one_minus_gamma_down;    /* the same for the downlink compression Top_K_down(g); 0 when unidirectional */
+    double rho;                     /* level 2 only (else -1).  With a^q the vector worker q compressed and K = K_down:
+                                       unidirectional  || Top_K(sum_q p_q a^q) - sum_q p_q Top_K(a^q) || / || s sum_q p_q g^q ||
+                                       bidirectional   || Top_K(delta + sum_q p_q a^q) - Top_K(delta + sum_q p_q Top_K(a^q)) ||
+                                                       / || s sum_q p_q g^q ||   (delta: server memory before the step)
+                                       (the two gap assumptions of Section 3; s = alpha with TK_MODE_EF, else 1: the
+                                       step size cancels) */
 } tk_diag;
 /*   one_minus_gamma_up_host: NULL, or [N] doubles that receive the per-worker values. */
-int tk_set_diagnostics(tk_ctx* ctx, int on);
+int tk_set_diagnostics(tk_ctx* ctx, int level);
 int tk_diagnostics(tk_ctx* ctx, tk_diag* out, double* one_minus_gamma_up_host);
 
 /* Record device timestamps around the streaming selection pass of every `every`-th tk_step

@@ -42,7 +42,7 @@ class tk_stats(ctypes.Structure):
 class tk_diag(ctypes.Structure):
     _fields_ = [("nonzero_fraction", ctypes.c_double), ("union_fraction", ctypes.c_double),
                 ("compression_factor", ctypes.c_double), ("one_minus_gamma_up_max", ctypes.c_double),
-                ("one_minus_gamma_down", ctypes.c_double)]
+                ("one_minus_gamma_down", ctypes.c_double), ("rho", ctypes.c_double)]
 
 
 _lib = None
@@ -224,8 +224,9 @@ class Context:
         eo, do = (e.value - base) // 4, (dl.value - base) // 4
         return flat[eo:eo + self.N * self.d].view(self.N, self.d), flat[do:do + self.d]
 
-    def tk_set_diagnostics(self, on: bool) -> None:
-        _check(load().tk_set_diagnostics(self._h, 1 if on else 0), "tk_set_diagnostics")
+    def tk_set_diagnostics(self, level) -> None:
+        """0 = off, 1 = cheap diagnostics, 2 = also the gap constant (re-reads the gradients)."""
+        _check(load().tk_set_diagnostics(self._h, int(level)), "tk_set_diagnostics")
 
     def tk_diagnostics(self):
         """(tk_diag, per-worker 1 - gamma list) of the last step."""

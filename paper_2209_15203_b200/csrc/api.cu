@@ -9,6 +9,7 @@
 
 #include "aggregate.cuh"
 #include "common.cuh"
+#include "diag.cuh"
 #include "select.cuh"
 #include "sort.cuh"
 
@@ -201,6 +202,14 @@ struct tk_ctx {
     float* delta = nullptr;    // [d]
     SelectBufs down;           // selection over the dense server vector (1 row of d)
     int64_t ef_kdown = 0;      // largest K_down the attached buffers serve
+    // gap-constant diagnostics (tk_set_diagnostics level 2): own allocation
+    char* diag_mem = nullptr;
+    float* diag_Da = nullptr;  // [d] dense sum of the compensated vectors (+ delta)
+    float* diag_Z = nullptr;   // [d] scratch for sparse differences, zero at rest
+    double* diag_sums = nullptr;  // [0] = squared denominator, [1] = squared numerator
+    SelectBufs diag_sel;       // Top_K over diag_Da
+    int64_t diag_kdown = 0;
+    const uint2* diag_other_ef() const { return down.out; }
     // captured steps (tk_set_graph)
     struct StepKey {
         float* w; const float* g; float alpha; int mode; int64_t K_down; int force_general, diagnostics;
@@ -502,6 +511,45 @@ int run_sort(cudaStream_t stream, uint2* src, size_t stride, const u32* counts, 
 
 }  // namespace
 
+namespace {
+void drop_graphs(tk_ctx* c) {
+    for (int i = 0; i < c->n_graphs; ++i) cudaGraphExecDestroy(c->graphs[i].exec);
+    c->n_graphs = 0;
+}
+
+int diag_alloc(tk_ctx* c) {
+    if (c->diag_mem && c->diag_kdown >= c->K_down) return TK_OK;
+    drop_graphs(c);
+    if (c->diag_mem) {
+        cudaStreamSynchronize(c->stream);
+        cudaFree(c->diag_mem);
+        c->diag_mem = nullptr;
+    }
+    SelectLayout L = select_layout(1, c->d, c->K_down);
+    size_t vec = align_up((size_t)c->d * sizeof(float));
+    size_t bytes = 2 * vec + align_up(2 * sizeof(double)) + L.bytes;
+    if (cudaMalloc((void**)&c->diag_mem, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        c->diag_mem = nullptr;
+        return TK_ERR_ALLOC;
+    }
+    c->diag_Da = (float*)c->diag_mem;
+    c->diag_Z = (float*)(c->diag_mem + vec);
+    c->diag_sums = (double*)(c->diag_mem + 2 * vec);
+    c->diag_sel = bind(L, c->diag_mem + 2 * vec + align_up(2 * sizeof(double)));
+    c->diag_kdown = c->K_down;
+    if (cudaMemsetAsync(c->diag_Z, 0, vec, c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->diag_sums, 0, 2 * sizeof(double), c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->diag_sel.rs, 0, sizeof(RowState), c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->diag_sel.hist, 0, (size_t)kHistBins * sizeof(u32), c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return TK_OK;
+}
+}  // namespace
+
 // ---- C ABI --------------------------------------------------------------------------------------
 extern "C" {
 
@@ -612,11 +660,6 @@ bool step_args_ok(tk_ctx* c, float alpha, int mode) {
 
 namespace {
 int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode, bool timed);
-
-void drop_graphs(tk_ctx* c) {
-    for (int i = 0; i < c->n_graphs; ++i) cudaGraphExecDestroy(c->graphs[i].exec);
-    c->n_graphs = 0;
-}
 }  // namespace
 
 int tk_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, int mode) {
@@ -696,12 +739,45 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
     // ... and its last kernel threads every uplink entry onto its coordinate's chain (and, with
     // error memories, zeroes the sent entries in eps)
     const bool diag = c->diagnostics != 0;
+    const bool gap = c->diagnostics >= 2 && c->diag_mem && c->diag_kdown >= c->K_down;
+    const bool bidir = (mode & TK_MODE_BIDIR) != 0;
+    int rc = TK_OK;
+    if (gap) {
+        // before the memories change: the dense sums, and Top_K of (delta +) sum_q p_q a^q
+        if (cudaMemsetAsync(c->diag_sums, 0, 2 * sizeof(double), s) != cudaSuccess) return TK_ERR_CUDA;
+        DeviceInfo* di = nullptr;
+        rc = device_info(&di);
+        if (rc != TK_OK) return rc;
+        dense_sums_kernel<<<di->sms * 8, 256, 0, s>>>(grads_dev, with_ef ? c->eps : nullptr,
+                                                      (with_ef && bidir) ? c->delta : nullptr, c->p, c->N, (size_t)c->d,
+                                                      alpha, with_ef ? alpha : 1.0f, c->diag_Da, c->diag_sums);
+        TK_LAUNCH_CHECK();
+        c->launches += 1;
+        rc = run_select(s, c->diag_Da, 1, c->d, c->K_down, c->diag_sel, c->ctrl, c->force_general != 0, nullptr,
+                        nullptr, &c->launches);
+        if (rc != TK_OK) return rc;
+    }
     LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0};
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
-    int rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
-                        &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
+    rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
+                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
     if (rc != TK_OK) return rc;
-    return run_server(c, w_dev, alpha, mode);
+    rc = run_server(c, w_dev, alpha, mode);
+    if (rc != TK_OK || !gap) return rc;
+    // after the step: the other side of the difference is what the server actually sent
+    const uint2* other = c->U;                      // unidirectional: S over the union
+    const u32* other_count = &c->uni->cand_count;
+    u32 other_cap = c->ucap;
+    if (bidir && with_ef) { other = c->diag_other_ef(); other_count = nullptr; other_cap = (u32)c->K_down; }
+    else if (bidir) { other = c->sel; other_count = &c->uni->out_count; other_cap = c->ucap; }
+    u32 Kd = (u32)c->K_down, dd = (u32)c->d;
+    diff_scatter_kernel<<<(Kd + 255) / 256, 256, 0, s>>>(c->diag_sel.out, nullptr, Kd, 1.0f, c->diag_Z, dd);
+    diff_scatter_kernel<<<(other_cap + 255) / 256, 256, 0, s>>>(other, other_count, other_cap, -1.0f, c->diag_Z, dd);
+    diff_norm_kernel<<<(Kd + 255) / 256, 256, 0, s>>>(c->diag_sel.out, nullptr, Kd, c->diag_Z, dd, c->diag_sums);
+    diff_norm_kernel<<<(other_cap + 255) / 256, 256, 0, s>>>(other, other_count, other_cap, c->diag_Z, dd, c->diag_sums);
+    TK_LAUNCH_CHECK();
+    c->launches += 4;
+    return TK_OK;
 }
 }  // namespace
 
@@ -830,6 +906,7 @@ int tk_ef_state(tk_ctx* c, float** eps_dev, float** delta_dev) {
 int tk_set_kdown(tk_ctx* c, int64_t K_down) {
     if (!c || K_down < 1 || K_down > c->d) return TK_ERR_INVALID;
     c->K_down = K_down;
+    if (c->diagnostics >= 2) return diag_alloc(c);   // the dense selection of the diagnostics grows with K_down
     return TK_OK;
 }
 
@@ -985,9 +1062,13 @@ int tk_set_profile(tk_ctx* c, int on) {
     return TK_OK;
 }
 
-int tk_set_diagnostics(tk_ctx* c, int on) {
-    if (!c) return TK_ERR_INVALID;
-    c->diagnostics = on ? 1 : 0;
+int tk_set_diagnostics(tk_ctx* c, int level) {
+    if (!c || level < 0 || level > 2) return TK_ERR_INVALID;
+    if (level == 2) {
+        int rc = diag_alloc(c);
+        if (rc != TK_OK) return rc;
+    }
+    c->diagnostics = level;
     return TK_OK;
 }
 
@@ -1029,6 +1110,15 @@ int tk_diagnostics(tk_ctx* c, tk_diag* out, double* one_minus_gamma_up_host) {
     out->compression_factor = (double)c->last_kdown / ((double)c->K_up * (double)c->N);
     if (ef_bidir) out->one_minus_gamma_down = lost(dn.sum_sq, dn.sel_sq);
     else if (c->last_mode & TK_MODE_BIDIR) out->one_minus_gamma_down = lost(u.sum_sq, u.sel_sq);
+    out->rho = -1.0;
+    if (c->diagnostics >= 2 && c->diag_mem) {
+        double sums[2] = {0.0, 0.0};
+        if (cudaMemcpy(sums, c->diag_sums, sizeof sums, cudaMemcpyDeviceToHost) != cudaSuccess) {
+            cudaGetLastError();
+            return TK_ERR_CUDA;
+        }
+        out->rho = sums[0] > 0.0 ? sqrt(sums[1]) / sqrt(sums[0]) : 0.0;
+    }
     return TK_OK;
 }
 
@@ -1054,6 +1144,7 @@ void tk_destroy(tk_ctx* c) {
         for (int i = 0; i < 2 * kMaxEvents; ++i) cudaEventDestroy(c->ev[i]);
     if (c->stage_g) cudaFree(c->stage_g);
     if (c->stage_w) cudaFree(c->stage_w);
+    if (c->diag_mem) cudaFree(c->diag_mem);
     delete c;
 }
 

@@ -175,7 +175,7 @@ def test_diagnostics_match_the_oracle():
         p = W.make_p(wl)
         K_down = wl.K_down[0]
         ctx = make_ctx(wl, K_down)
-        ctx.tk_set_diagnostics(True)
+        ctx.tk_set_diagnostics(1)
         if ef:
             ctx.tk_ef_attach()
         w = W.make_w(wl, DEV)
@@ -240,6 +240,43 @@ def test_graph_replay_matches_direct_launches():
         ia, va = direct.tk_last_downlink()
         ib, vb = graphed.tk_last_downlink()
         assert torch.equal(ia, ib) and torch.equal(va.view(torch.int32), vb.view(torch.int32))
+
+
+@pytest.mark.parametrize("ef", [False, True])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_gap_constant_matches_the_oracle(mode, ef):
+    # rho_hat (unidirectional) / rho (bidirectional) of every step, memories carried along
+    for wl in (W.workload(2, d=400_000, N=4), W.workload(1, d=20_000)):
+        p = W.make_p(wl)
+        K_down = wl.K_down[0]
+        ctx = make_ctx(wl, K_down)
+        if ef:
+            ctx.tk_ef_attach()
+        ctx.tk_set_diagnostics(2)
+        w = W.make_w(wl, DEV)
+        w_ref = w.cpu().numpy()
+        eps = np.zeros((wl.N, wl.d), np.float32)
+        delta = np.zeros(wl.d, np.float32)
+        for s in range(3):
+            G = W.make_grads(wl, s, DEV)
+            Gh = G.cpu().numpy()
+            ctx.tk_step(w, G, wl.alpha, mode | (binding.TK_MODE_EF if ef else 0))
+            diag, _ = ctx.tk_diagnostics()
+            if ef:
+                want = oracle.ref_rho(Gh, eps, delta if mode == 1 else None, wl.K_up, K_down, p.numpy(), wl.alpha, mode)
+                ref = oracle.ref_step_ef(w_ref, eps, delta, Gh, wl.K_up, K_down, p.numpy(), wl.alpha, mode)
+                eps = ref.eps
+                if mode == 1:
+                    delta = ref.delta
+            else:
+                want = oracle.ref_rho(Gh, None, None, wl.K_up, K_down, p.numpy(), wl.alpha, mode)
+                ref = oracle.ref_step(w_ref, Gh, wl.K_up, K_down, p.numpy(), wl.alpha, mode)
+            w_ref = ref.w
+            assert want > 0
+            assert abs(diag.rho - want) <= 1e-5 * want, (mode, ef, s, diag.rho, want)
+            assert_values_close(w.cpu().numpy(), ref.w, "w with diagnostics on")
+        assert ctx.tk_status().device_status == 0
+        ctx.close()
 
 
 def test_bad_arguments_are_rejected():
