@@ -97,6 +97,44 @@ def test_student_dirichlet_many_steps():
     run_ef(W.workload(3, d=700_000, N=5), 6, 1)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_toy_example_trajectory(mode):
+    # the paper's toy example (appendix): three quadratics in R^100, K = 1, alpha = 0.01; 300
+    # iterations with the gradients taken at the current w, GPU and oracle side by side
+    d, N = 100, 3
+    centres = np.array([1.0, 5.0, 10.0], np.float32)
+    p = torch.full((N,), 1.0 / 3.0)
+    np.random.seed(10)
+    w_ref = np.random.normal(20, 1, d).astype(np.float32)
+    ctx = binding.Context(d, N, 1, 1, p)
+    ctx.tk_ef_attach()
+    ctx.tk_set_diagnostics(2)
+    w_dev = torch.from_numpy(w_ref.copy()).to(DEV)
+    c_dev = torch.from_numpy(centres).to(DEV)
+    eps = np.zeros((N, d), np.float32)
+    delta = np.zeros(d, np.float32)
+    rhos = []
+    for t in range(300):
+        G = (w_dev[None, :] - c_dev[:, None]).contiguous()
+        Gh = (w_ref[None, :] - centres[:, None]).astype(np.float32)
+        assert np.array_equal(G.cpu().numpy(), Gh)
+        ctx.tk_step(w_dev, G, 0.01, mode | EF)
+        ref = oracle.ref_step_ef(w_ref, eps, delta, Gh, 1, 1, p.numpy(), 0.01, mode)
+        w_ref, eps = ref.w, ref.eps
+        if mode == 1:
+            delta = ref.delta
+        if t % 50 == 49:
+            assert np.array_equal(w_dev.cpu().numpy().view(np.uint32), w_ref.view(np.uint32)), "w diverged at t=%d" % t
+            rhos.append(ctx.tk_diagnostics()[0].rho)
+    e_dev, d_dev = ctx.tk_ef_state()
+    assert np.array_equal(e_dev.cpu().numpy().view(np.uint32), eps.view(np.uint32))
+    if mode == 1:
+        assert np.array_equal(d_dev.cpu().numpy().view(np.uint32), delta.view(np.uint32))
+    assert ctx.tk_status().device_status == 0 and all(r >= 0 for r in rhos)
+    F = sum(0.5 * np.sum((w_ref.astype(np.float64) - c) ** 2) for c in (1.0, 5.0, 10.0)) / 3
+    assert 6100 / 9 < F < 6100 / 9 + 40          # hovers near F* = 6100/9, as the paper describes
+
+
 def test_needs_attached_memories():
     wl = W.workload(1, d=2000)
     ctx = binding.Context(wl.d, wl.N, wl.K_up, wl.K_up, W.make_p(wl))
