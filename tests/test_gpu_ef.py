@@ -172,3 +172,41 @@ def test_full_size_configs_with_memories(cid, steps):
     if psutil.virtual_memory().available < wl.N * wl.d * 4 * 6 + 16 * wl.d * 8:
         pytest.skip("not enough host memory for the oracle at this size")
     run_ef(wl, steps, 1)
+
+
+def test_random_small_problems_with_memories():
+    # many small shapes (every row alignment, tiny and large K, K_down above and below the union),
+    # five steps each with the memories carried along
+    rng = np.random.default_rng(915203)
+    for case in range(16):
+        N = int(rng.integers(1, 7))
+        d = int(rng.integers(8, 30_000))
+        K_up = int(rng.integers(1, max(2, d // 20)))
+        K_down = int(rng.integers(1, min(d, 3 * N * K_up) + 1))
+        mode = int(rng.integers(0, 2))
+        p = torch.from_numpy(rng.dirichlet(np.ones(N)).astype(np.float32))
+        ctx = binding.Context(d, N, K_up, K_down, p)
+        ctx.tk_ef_attach()
+        w_dev = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+        w = w_dev.cpu().numpy()
+        eps = np.zeros((N, d), np.float32)
+        delta = np.zeros(d, np.float32)
+        for s in range(5):
+            Gh = (rng.standard_t(3, (N, d)) * 1e-2).astype(np.float32)
+            if case % 3 == 0:
+                Gh = np.round(Gh * 64) / 64                      # coarse values: many ties
+            G = torch.from_numpy(Gh.astype(np.float32)).to(DEV)
+            ctx.tk_step(w_dev, G, 0.25, mode | EF)
+            ref = oracle.ref_step_ef(w, eps, delta, Gh, K_up, K_down, p.numpy(), 0.25, mode)
+            what = "case %d (N=%d d=%d K=%d/%d mode=%d) step %d" % (case, N, d, K_up, K_down, mode, s)
+            midx, _ = ctx.tk_last_downlink()
+            assert np.array_equal(midx.cpu().numpy(), ref.msg_idx), what
+            assert_values_close(w_dev.cpu().numpy(), ref.w, what + " w")
+            e_dev, d_dev = ctx.tk_ef_state()
+            assert_values_close(e_dev.cpu().numpy(), ref.eps, what + " epsilon")
+            if mode == 1:
+                assert_values_close(d_dev.cpu().numpy(), ref.delta, what + " delta")
+                delta = ref.delta
+            w, eps = ref.w, ref.eps
+        assert ctx.tk_status().device_status == 0
+        ctx.close()
