@@ -142,6 +142,24 @@ def test_cancelling_workers_and_zero_weights():
                        "cancel p=%s mode=%d" % (p, mode))
 
 
+@pytest.mark.parametrize("N,d,K_up,K_down", [(5000, 2003, 3, 40), (65535, 4001, 2, 300)])
+def test_many_workers(N, d, K_up, K_down):
+    # more workers than one selection launch takes (4096), and the largest N the ABI accepts
+    rng = np.random.default_rng(N)
+    G = torch.from_numpy(rng.standard_normal((N, d)).astype(np.float32)).to(DEV)
+    p = torch.from_numpy((rng.random(N) / N).astype(np.float32))
+    wl = W.workload(1, d=d, N=N)
+    wl = wl.__class__(**{**wl.__dict__, "K_up": K_up, "K_down": (K_down,)})
+    for mode in (0, 1):
+        ctx = binding.Context(d, N, K_up, K_down, p)
+        _P[id(ctx)] = p.numpy()
+        w_dev = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+        w_ref = w_dev.cpu().numpy()
+        for s in range(2):
+            w_ref = check_step(ctx, wl, w_dev, w_ref, G, 0.05, mode, K_down, "N=%d mode=%d step=%d" % (N, mode, s))
+        ctx.close()
+
+
 def test_step_host_matches_device_step():
     wl = W.workload(2, d=500_000, N=4)
     G = W.make_grads(wl, 0, DEV)

@@ -160,6 +160,26 @@ def test_random_shapes_sweep():
         run_both(x.astype(np.float32), K)
 
 
+def test_more_rows_than_one_launch_takes():
+    # rows are processed in batches of 4096: short rows (multi-pass path) across two batch boundaries
+    rng = np.random.default_rng(77)
+    run_both(rng.standard_normal((9000, 301)).astype(np.float32), 7)
+    # ... and rows just long enough for the sampled path (its many-rows variant); the oracle checks
+    # a sample of the rows, among them the ones on either side of the batch boundary
+    rows, d, K = 4200, 131_102, 100
+    g = torch.Generator(device=DEV)
+    g.manual_seed(78)
+    x = torch.randn((rows, d), generator=g, device=DEV, dtype=torch.float32)
+    idx, val = binding.tk_topk(x, K)
+    torch.cuda.synchronize()
+    pick = np.unique(np.concatenate([[0, 1, 4094, 4095, 4096, 4097, rows - 1], rng.integers(0, rows, 40)]))
+    ridx, rval = oracle.ref_topk_rows(x[torch.from_numpy(pick).to(DEV)].cpu().numpy(), K)
+    assert_message_equal(idx[pick], val[pick], ridx, rval, "tk_topk 4200 rows (sampled rows)")
+    # all rows: the selected magnitudes are the K largest of the row (torch.topk on |x|, values only)
+    top = torch.topk(x.abs(), K, dim=1).values.sort(dim=1).values
+    assert torch.equal(val.abs().sort(dim=1).values, top)
+
+
 def test_argument_errors():
     x = torch.zeros(100, device=DEV)
     with pytest.raises(binding.TkError):
