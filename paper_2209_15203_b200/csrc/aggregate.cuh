@@ -5,7 +5,7 @@
 // steps) is the scatter target: the uplink selection, as it emits entry number
 // e = q*K_up + slot with coordinate j, threads it onto j's chain
 // (next[e] = exchange(head[j], e+1), see emit_entry); agg_reduce lets the entry at the
-// head of each chain walk it in ascending worker order, accumulate
+// head of each chain gather the chain's entries and, in ascending worker order, accumulate
 //        g_j = fl(g_j + fl(p_q * v_{q,j}))        starting from +0,
 // append (j, g_j) to the union list U, put the word back to zero, and — in
 // unidirectional mode, where the downlink carries g itself — apply
@@ -34,6 +34,9 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, R
     next[e] = atomicExch(&head[j], e + 1);
 }
 
+constexpr int kChainKeep = 128;  // entries of a coordinate's chain remembered from the first walk
+constexpr int kWindow = 64;      // consecutive workers whose terms one round adds
+
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
                   u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
@@ -49,19 +52,51 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         owner = j < d && __ldcg(&head[j]) == e + 1;
     }
     if (owner) {
-        // walk the chain once per term, each time taking the smallest worker not yet added
-        int last_q = -1;
-        for (u32 guard = 0; guard <= total; ++guard) {
-            int best_q = 0x7fffffff;
-            u32 best_e = 0;
-            for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) {
-                int q = (int)((c - 1) / K_up);
-                if (q > last_q && q < best_q) { best_q = q; best_e = c - 1; }
+        // Entry ids grow with the worker (e = q*K_up + slot) and a worker sends a coordinate at most
+        // once.  The chain is walked once (a string of dependent loads: the expensive part) and its
+        // first kChainKeep entries are kept; the terms are then added in rounds, each taking the
+        // workers of one window of kWindow consecutive numbers in order (a bit mask says which of them
+        // sent the coordinate, a small table where their entries are).  Only a chain longer than
+        // kChainKeep is walked again, once per round.
+        u32 ids[kChainKeep];
+        u32 byq[kWindow];
+        u32 L = 0, min_id = 0xffffffffu;
+        for (u32 c = e + 1; c != 0 && L <= total; c = next[c - 1]) {
+            if (L < (u32)kChainKeep) ids[L] = c - 1;
+            min_id = min(min_id, c - 1);
+            ++L;
+        }
+        if (L == 1) {
+            acc = __fadd_rn(acc, __fmul_rn(p[e / K_up], __uint_as_float(up[e].y)));
+        } else {
+            const bool kept = L <= (u32)kChainKeep;
+            u32 qlo = min_id / K_up;  // workers below qlo are done
+            for (u32 guard = 0; guard <= total; ++guard) {
+                u64 mask = 0;
+                u32 qnext = 0xffffffffu;
+                auto visit = [&](u32 id) {
+                    u32 q = id / K_up;
+                    if (q < qlo) return;
+                    if (q - qlo < (u32)kWindow) {
+                        byq[q - qlo] = id;
+                        mask |= 1ull << (q - qlo);
+                    } else {
+                        qnext = min(qnext, q);
+                    }
+                };
+                if (kept) {
+                    for (u32 k = 0; k < L; ++k) visit(ids[k]);
+                } else {
+                    for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) visit(c - 1);
+                }
+                while (mask) {
+                    int b = __ffsll((long long)mask) - 1;
+                    mask &= mask - 1;
+                    acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(up[byq[b]].y)));
+                }
+                if (qnext == 0xffffffffu) break;
+                qlo = qnext;
             }
-            if (best_q == 0x7fffffff) break;
-            float term = __fmul_rn(p[best_q], __uint_as_float(up[best_e].y));
-            acc = __fadd_rn(acc, term);
-            last_q = best_q;
         }
         head[j] = 0;
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));

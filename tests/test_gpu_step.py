@@ -160,6 +160,28 @@ def test_many_workers(N, d, K_up, K_down):
         ctx.close()
 
 
+@pytest.mark.parametrize("N,noise", [(20, 0.01), (100, 0.01), (150, 0.0)])
+def test_workers_that_agree(N, noise):
+    # correlated gradients: almost every selected coordinate is sent by all N workers, so the sums
+    # have N terms (more than one window of workers, and with N = 150 more than the server step
+    # remembers from its first walk of a chain)
+    d, K = 60_002, 300
+    rng = np.random.default_rng(1000 + N)
+    base = rng.standard_normal(d)
+    G = torch.from_numpy((base[None, :] * (1.0 + noise * rng.standard_normal((N, d)))).astype(np.float32)).to(DEV)
+    p = torch.from_numpy((rng.random(N) + 0.5).astype(np.float32) / N)
+    wl = W.workload(1, d=d, N=N)
+    wl = wl.__class__(**{**wl.__dict__, "K_up": K, "K_down": (K,)})
+    for mode in (0, 1):
+        ctx = binding.Context(d, N, K, K, p)
+        _P[id(ctx)] = p.numpy()
+        w_dev = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+        w_ref = check_step(ctx, wl, w_dev, w_dev.cpu().numpy(), G, 0.05, mode, K, "agreeing workers N=%d mode=%d" % (N, mode))
+        assert ctx.tk_status().union_size < 2 * K
+        check_step(ctx, wl, w_dev, w_ref, G, 0.05, mode, K, "agreeing workers N=%d mode=%d step 2" % (N, mode))
+        ctx.close()
+
+
 def test_step_host_matches_device_step():
     wl = W.workload(2, d=500_000, N=4)
     G = W.make_grads(wl, 0, DEV)
