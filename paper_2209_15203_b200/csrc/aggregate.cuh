@@ -34,8 +34,7 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, R
     next[e] = atomicExch(&head[j], e + 1);
 }
 
-constexpr int kChainKeep = 128;  // entries of a coordinate's chain remembered from the first walk
-constexpr int kWindow = 64;      // consecutive workers whose terms one round adds
+constexpr int kWindow = 128;  // consecutive workers whose terms one walk of a chain gathers (two 64-bit masks)
 
 __global__ void __launch_bounds__(256)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
@@ -53,50 +52,51 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     }
     if (owner) {
         // Entry ids grow with the worker (e = q*K_up + slot) and a worker sends a coordinate at most
-        // once.  The chain is walked once (a string of dependent loads: the expensive part) and its
-        // first kChainKeep entries are kept; the terms are then added in rounds, each taking the
-        // workers of one window of kWindow consecutive numbers in order (a bit mask says which of them
-        // sent the coordinate, a small table where their entries are).  Only a chain longer than
-        // kChainKeep is walked again, once per round.
-        u32 ids[kChainKeep];
-        u32 byq[kWindow];
-        u32 L = 0, min_id = 0xffffffffu;
-        for (u32 c = e + 1; c != 0 && L <= total; c = next[c - 1]) {
-            if (L < (u32)kChainKeep) ids[L] = c - 1;
-            min_id = min(min_id, c - 1);
-            ++L;
+        // once.  A walk of the chain is a string of dependent loads, the expensive part; each hop
+        // also fetches the entry's value, so the two latencies overlap.  The values of the workers
+        // in a window of kWindow consecutive numbers go into a small table with a bit mask saying
+        // which are present; the terms are then added in ascending worker order.  With at most
+        // kWindow workers that is a single walk; with more, one walk finds the first sender and
+        // one walk per window that has senders follows.
+        u32 byv[kWindow];
+        u32 qlo = 0;  // workers below qlo are done
+        if (total > (u32)kWindow * K_up) {
+            u32 min_id = e;
+            for (u32 c = next[e], hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) min_id = min(min_id, c - 1);
+            qlo = min_id / K_up;
         }
-        if (L == 1) {
-            acc = __fadd_rn(acc, __fmul_rn(p[e / K_up], __uint_as_float(up[e].y)));
-        } else {
-            const bool kept = L <= (u32)kChainKeep;
-            u32 qlo = min_id / K_up;  // workers below qlo are done
-            for (u32 guard = 0; guard <= total; ++guard) {
-                u64 mask = 0;
-                u32 qnext = 0xffffffffu;
-                auto visit = [&](u32 id) {
-                    u32 q = id / K_up;
-                    if (q < qlo) return;
-                    if (q - qlo < (u32)kWindow) {
-                        byq[q - qlo] = id;
-                        mask |= 1ull << (q - qlo);
+        for (u32 guard = 0; guard <= total; ++guard) {
+            u64 m0 = 0, m1 = 0;
+            u32 qnext = 0xffffffffu;
+            for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; ++hops) {
+                const u32 id = c - 1;
+                const u32 nx = next[id];
+                const u32 v = up[id].y;
+                const u32 q = id / K_up;
+                if (q >= qlo) {
+                    const u32 o = q - qlo;
+                    if (o < (u32)kWindow) {
+                        byv[o] = v;
+                        if (o < 64u) m0 |= 1ull << o;
+                        else m1 |= 1ull << (o - 64u);
                     } else {
                         qnext = min(qnext, q);
                     }
-                };
-                if (kept) {
-                    for (u32 k = 0; k < L; ++k) visit(ids[k]);
-                } else {
-                    for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) visit(c - 1);
                 }
-                while (mask) {
-                    int b = __ffsll((long long)mask) - 1;
-                    mask &= mask - 1;
-                    acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(up[byq[b]].y)));
-                }
-                if (qnext == 0xffffffffu) break;
-                qlo = qnext;
+                c = nx;
             }
+            while (m0) {
+                const int b = __ffsll((long long)m0) - 1;
+                m0 &= m0 - 1;
+                acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
+            }
+            while (m1) {
+                const int b = __ffsll((long long)m1) + 63;
+                m1 &= m1 - 1;
+                acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
+            }
+            if (qnext == 0xffffffffu) break;
+            qlo = qnext;
         }
         head[j] = 0;
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
