@@ -130,7 +130,7 @@ def run_reference(args, rank, world):
     K_down = wl.K_down[0]
     times = []
     for s in range(total_steps):
-        G = W.make_grads(wl, s, "cpu", scale=scale).numpy()
+        G = W.make_grads(wl, s, "cpu", scale=scale, agree=args.agree).numpy()
         t0 = time.perf_counter()
         res = oracle.ref_step(w, G, wl.K_up, K_down, p, wl.alpha, 1, nthreads=threads, want_dense=False)
         t1 = time.perf_counter()
@@ -172,6 +172,9 @@ def main():
                     "replaying captured CUDA graphs (tk_set_graph)")
     ap.add_argument("--profile-every", type=int, default=4, help="timestamp the streaming kernel of every n-th timed "
                     "step (such a step is issued as plain launches)")
+    ap.add_argument("--agree", type=float, default=None, metavar="C",
+                    help="workers see noisy copies of one shared vector, row_q = base * (1 + C z_q), instead of "
+                         "independent rows: their selections then mostly coincide (union near K)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -207,7 +210,7 @@ def main():
     ctx = binding.Context(wl.d, wl.N, wl.K_up, K_down, p, stream=run_stream)
     scale = W.scale_vector(wl, dev)
     nbuf = max(1, min(args.steps, 8))
-    bufs = [W.make_grads(wl, s, dev, scale=scale) for s in range(nbuf)]
+    bufs = [W.make_grads(wl, s, dev, scale=scale, agree=args.agree) for s in range(nbuf)]
     del scale
     w = W.make_w(wl, dev)
     mode = binding.TK_MODE_BIDIR | (binding.TK_MODE_EF if args.ef else 0)
@@ -324,6 +327,8 @@ def main():
                                "streaming kernel" % max(1, args.profile_every)) if args.graph else "stream launches",
                     "parallelism": ("workers sharded over %d ranks, one all-gather per step" if args.sharded
                                     else "replicas x%d") % world})
+        if args.agree is not None:
+            cfg["rows"] = "shared vector x (1 + %g z_q)" % args.agree
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,

@@ -191,13 +191,29 @@ def _plant(wl: Workload, G: torch.Tensor, step: int, device) -> None:
 
 
 def make_grads(wl: Workload, step: int, device, out: Optional[torch.Tensor] = None,
-               scale: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """The N workers' vectors for one step, fp32 [N][d] on ``device``."""
+               scale: Optional[torch.Tensor] = None, agree: Optional[float] = None) -> torch.Tensor:
+    """The N workers' vectors for one step, fp32 [N][d] on ``device``.
+
+    By default the rows are drawn independently.  With ``agree`` = c the workers see noisy
+    copies of one shared vector, row_q = base * (1 + c * z_q) with z_q standard normal, the way
+    workers that sample the same loss do: their K largest coordinates then mostly coincide."""
     seed = BASE_SEED + 10007 * wl.cid + step
     g = _gen(device, seed)
     G = out if out is not None else torch.empty((wl.N, wl.d), device=device, dtype=torch.float32)
     if scale is None:
         scale = scale_vector(wl, device)
+    if agree is not None:
+        base = _student_row(wl.d, g, device) if wl.dist == "student" else \
+            torch.randn(wl.d, generator=g, device=device, dtype=torch.float32)
+        base *= scale if scale is not None else wl.sigma_lo
+        for q in range(wl.N):
+            z = torch.randn(wl.d, generator=g, device=device, dtype=torch.float32)
+            z.mul_(agree).add_(1.0).mul_(base)
+            G[q].copy_(z)
+            del z
+        if wl.adversarial:
+            _plant(wl, G, step, device)
+        return G
     for q in range(wl.N):
         if wl.dist == "student":
             row = _student_row(wl.d, g, device)

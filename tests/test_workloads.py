@@ -54,3 +54,16 @@ def test_adversarial_rows_have_zeros_and_straddling_ties():
     # paired workers carry the planted magnitudes with opposite signs
     both = (np.abs(G[0]) == np.abs(G[1])) & (G[0] != 0)
     assert both.sum() >= 1500 and np.all(G[0][both] == -G[1][both])
+
+
+def test_agreeing_workers_share_their_large_coordinates():
+    wl = W.workload(2, d=200_000, N=6)
+    A = W.make_grads(wl, 0, "cpu", agree=0.01)
+    B = W.make_grads(wl, 0, "cpu", agree=0.01)
+    assert torch.equal(A, B)
+    assert not torch.equal(A, W.make_grads(wl, 0, "cpu"))          # the default rows are independent draws
+    top = [set(torch.topk(A[q].abs(), wl.K_up).indices.tolist()) for q in range(wl.N)]
+    common = set.intersection(*top)
+    assert len(common) > 0.7 * wl.K_up
+    ratio = A[1] / A[0]
+    assert 0.005 < float(ratio[torch.isfinite(ratio)].std()) < 0.03
