@@ -2,13 +2,27 @@
 // worker order so that the fp32 result does not depend on scheduling.
 //
 // The dense server buffer (one 32-bit word per coordinate, all zero between
-// steps) is the scatter target: the uplink selection, as it emits entry number
-// e = q*K_up + slot with coordinate j, threads it onto j's chain
-// (next[e] = exchange(head[j], e+1), see emit_entry); agg_reduce lets the entry at the
-// head of each chain gather the chain's entries and, in ascending worker order, accumulate
+// steps) is the scatter target.  Entry number e = q*K_up + slot of the uplink
+// messages carries (coordinate j, value v) of worker q; the uplink selection
+// files it under j as it emits it (see emit_entry), in one of two ways:
+//
+//   slots   (at most kSlotWorkers workers and a slot table that fits the budget)
+//           head[j] keeps the first entry e0 to arrive: it owns the coordinate.
+//           Every later entry sets the word's top bit ("shared"), sets its worker's
+//           bit in the 128-bit mask at the start of row e0 of the table and writes
+//           its value to its worker's column of that row.  agg_reduce: an owner
+//           whose coordinate is not shared has the whole sum in its own entry; a
+//           shared one reads the mask and then the columns it names — independent
+//           loads, eight at a time — and adds them, its own value at its own
+//           worker's place, in worker order.
+//   chains  (otherwise)  next[e] = exchange(head[j], e+1); the entry at the head
+//           of a chain walks it — dependent loads, one per sender — and puts
+//           the terms in worker order.
+//
+// Either way the owner accumulates
 //        g_j = fl(g_j + fl(p_q * v_{q,j}))        starting from +0,
-// append (j, g_j) to the union list U, put the word back to zero, and — in
-// unidirectional mode, where the downlink carries g itself — apply
+// appends (j, g_j) to the union list U, puts the words it used back to zero, and
+// — in unidirectional mode, where the downlink carries g itself — applies
 // w_j <- w_j - alpha g_j  right there (last worker step of Algorithm 1).
 // With the server memory of Algorithm 2 it adds the sum into delta instead.
 // The work is O(N K_up); no pass over the d coordinates is ever made.
@@ -21,8 +35,11 @@ namespace tk {
 // Threads every entry of a gathered message buffer onto its coordinate's chain — what the
 // uplink selection's emission does on the fly when the messages are produced on this GPU.
 // Also resets the union's state for the step.
+constexpr int kSlotWorkers = 128;  // the slot table is used up to this many workers
+
 __global__ void __launch_bounds__(256)
-agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, RowState* uni, Ctrl* ctrl, u32 d) {
+agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u32* next, u32* slots, u32 row_words,
+                RowState* uni, Ctrl* ctrl, u32 d) {
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) {
         uni->lo = 0; uni->cand_count = 0; uni->max_key = 0; uni->out_count = 0; uni->flags = 0;
@@ -31,26 +48,67 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32* head, u32* next, R
     if (e >= total) return;
     u32 j = up[e].x;
     if (j >= d) { raise_status(ctrl, -5); next[e] = 0; return; }
-    next[e] = atomicExch(&head[j], e + 1);
+    if (slots) {
+        file_in_slot(head, slots, row_words, atomicCAS(&head[j], 0u, e + 1), j, e / K_up, up[e].y);
+    } else {
+        next[e] = atomicExch(&head[j], e + 1);
+    }
 }
 
 constexpr int kWindow = 128;  // consecutive workers whose terms one walk of a chain gathers (two 64-bit masks)
 
-__global__ void __launch_bounds__(256)
+// (256, 8): all 2048 threads of an SM stay resident — the kernel lives on memory parallelism
+__global__ void __launch_bounds__(256, 8)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
-                  u32* head, const u32* __restrict__ next, RowState* uni /* the union's state */,
+                  u32* head, const u32* __restrict__ next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
                   int stats) {
     dependency_wait();   // the chains are built by the kernel before
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
-    u32 j = 0;
+    u32 j = 0, own_bits = 0;
     float acc = 0.0f;
+    bool shared = false;
     if (e < total) {
-        j = up[e].x;
-        owner = j < d && __ldcg(&head[j]) == e + 1;
+        uint2 mine = up[e];
+        j = mine.x;
+        own_bits = mine.y;
+        u32 h = j < d ? __ldcg(&head[j]) : 0u;
+        // with chains the word is a plain entry number (N*K_up < 2^31), so the mask changes nothing
+        owner = (h & 0x7fffffffu) == e + 1;
+        shared = (h >> 31) != 0;
     }
-    if (owner) {
+    if (owner && slots) {
+        const u32 own_q = e / K_up;
+        if (!shared) {
+            acc = __fadd_rn(acc, __fmul_rn(p[own_q], __uint_as_float(own_bits)));
+        } else {
+            u32* row = slots + (size_t)e * row_words;
+            const uint4 m = __ldcg(reinterpret_cast<const uint4*>(row));
+            u64 m0 = (u64)m.x | ((u64)m.y << 32), m1 = (u64)m.z | ((u64)m.w << 32);
+            if (own_q < 64u) m0 |= 1ull << own_q;
+            else m1 |= 1ull << (own_q - 64u);
+            while (m0 | m1) {
+                u32 qs[8], vs[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {  // the next eight senders, their values all requested at once
+                    qs[i] = 0xffffffffu;
+                    if (m0) { qs[i] = (u32)__ffsll((long long)m0) - 1u; m0 &= m0 - 1; }
+                    else if (m1) { qs[i] = (u32)__ffsll((long long)m1) + 63u; m1 &= m1 - 1; }
+                    vs[i] = 0;
+                    if (qs[i] == own_q) vs[i] = own_bits;
+                    else if (qs[i] != 0xffffffffu) vs[i] = __ldcg(row + kSlotMaskWords + qs[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (qs[i] == 0xffffffffu) continue;
+                    acc = __fadd_rn(acc, __fmul_rn(p[qs[i]], __uint_as_float(vs[i])));
+                    if (qs[i] != own_q) row[kSlotMaskWords + qs[i]] = 0;
+                }
+            }
+            *reinterpret_cast<uint4*>(row) = make_uint4(0, 0, 0, 0);
+        }
+    } else if (owner) {  // chains
         // Entry ids grow with the worker (e = q*K_up + slot) and a worker sends a coordinate at most
         // once.  A walk of the chain is a string of dependent loads, the expensive part; each hop
         // also fetches the entry's value, so the two latencies overlap.  The values of the workers
@@ -98,6 +156,8 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
             if (qnext == 0xffffffffu) break;
             qlo = qnext;
         }
+    }
+    if (owner) {
         head[j] = 0;
         if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
         // server memory (Algorithm 2): g = sum + delta, kept in the memory until the downlink

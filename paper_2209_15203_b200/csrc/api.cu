@@ -180,6 +180,8 @@ struct tk_ctx {
     RowState* uni = nullptr;   // state of the union list / downlink selection
     u32* head = nullptr;       // [d] dense server buffer, zero at rest
     u32* next = nullptr;       // [N*K_up]
+    u32* slots = nullptr;      // [N*K_up][slot_row_words] slot table, zero at rest; NULL when the server step uses chains
+    u32 slot_row_words = 0;
     uint2* U = nullptr;        // [ucap] aggregate over the union
     uint2* sel = nullptr;      // [ucap] downlink message (unordered)
     u32* ghist = nullptr;      // [3][kHistBins] histograms of the grid-wide select, zero at rest
@@ -230,10 +232,17 @@ struct tk_ctx {
 namespace {
 
 struct CtxLayout {
-    size_t off_ctrl, off_p, off_sel_up, off_uni, off_head, off_next, off_U, off_sel, off_ghist, bytes;
+    size_t off_ctrl, off_p, off_sel_up, off_uni, off_head, off_next, off_slots, off_U, off_sel, off_ghist, bytes;
+    size_t slot_words;  // 0: the server step uses chains
+    u32 slot_row_words;
     SelectLayout up;
     u32 ucap;
 };
+
+#ifndef TK_SLOT_BUDGET
+#define TK_SLOT_BUDGET ((size_t)1 << 30)
+#endif
+constexpr size_t kSlotBudget = TK_SLOT_BUDGET;  // largest slot table of the server step, bytes (0: always chains)
 
 bool sizes_ok(int64_t d, int64_t N, int64_t K_up, int64_t K_down) {
     return d >= 1 && d < ((int64_t)1 << 31) && N >= 1 && N <= 65535 && K_up >= 1 && K_up <= d &&
@@ -252,6 +261,18 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
     L.off_uni = o;    o += align_up(sizeof(RowState));
     L.off_head = o;   o += align_up((size_t)d * sizeof(u32));
     L.off_next = o;   o += align_up((size_t)(N * K_up) * sizeof(u32));
+    // slot table of the server step: per uplink entry one row of a 128-bit mask plus one word per worker
+    // (rounded up to 16 bytes), when the workers are few and the table stays within kSlotBudget bytes
+    L.slot_row_words = 0;
+    L.slot_words = 0;
+    {
+        size_t row_words = kSlotMaskWords + (size_t)((N + 3) / 4 * 4);
+        if (N <= kSlotWorkers && row_words * (size_t)(N * K_up) * sizeof(u32) <= kSlotBudget) {
+            L.slot_row_words = (u32)row_words;
+            L.slot_words = row_words * (size_t)(N * K_up);
+        }
+    }
+    L.off_slots = o;  o += align_up(L.slot_words * sizeof(u32));
     L.off_U = o;      o += align_up((size_t)ucap * sizeof(uint2));
     L.off_sel = o;    o += align_up((size_t)ucap * sizeof(uint2));
     L.off_ghist = o;  o += align_up((size_t)3 * kHistBins * sizeof(u32));
@@ -583,6 +604,8 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
     c->uni = (RowState*)(c->ws + L.off_uni);
     c->head = (u32*)(c->ws + L.off_head);
     c->next = (u32*)(c->ws + L.off_next);
+    c->slots = L.slot_words ? (u32*)(c->ws + L.off_slots) : nullptr;
+    c->slot_row_words = L.slot_row_words;
     c->U = (uint2*)(c->ws + L.off_U);
     c->sel = (uint2*)(c->ws + L.off_sel);
     c->ghist = (u32*)(c->ws + L.off_ghist);
@@ -594,6 +617,7 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
               cudaMemsetAsync(c->uni, 0, sizeof(RowState), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->ghist, 0, (size_t)3 * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->head, 0, (size_t)d * sizeof(u32), c->stream) == cudaSuccess &&
+              (!c->slots || cudaMemsetAsync(c->slots, 0, L.slot_words * sizeof(u32), c->stream) == cudaSuccess) &&
               cudaMemcpyAsync(c->p, p_host, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream) ==
                   cudaSuccess &&
               cudaStreamSynchronize(c->stream) == cudaSuccess;
@@ -618,7 +642,8 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     u32 total = (u32)(c->N * c->K_up);
     u32 blocks = (total + 255) / 256;
     int rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(256), 0, s, 0, (const uint2*)c->up.out, total,
-                              (u32)c->K_up, (const float*)c->p, c->head, (const u32*)c->next, c->uni, c->U, c->ucap, w_dev,
+                              (u32)c->K_up, (const float*)c->p, c->head, (const u32*)c->next, c->slots, c->slot_row_words, c->uni, c->U,
+                              c->ucap, w_dev,
                               scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : (float*)nullptr, c->ctrl, (u32)c->d,
                               diag ? 1 : 0);
     if (rc != TK_OK) return rc;
@@ -757,7 +782,7 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
                         nullptr, &c->launches);
         if (rc != TK_OK) return rc;
     }
-    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0};
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0, c->slots, c->slot_row_words};
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
     rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
                     &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
@@ -809,8 +834,8 @@ int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {
 int tk_step_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     if (!step_args_ok(c, alpha, mode) || !aligned4(w_dev)) return TK_ERR_INVALID;
     u32 total = (u32)(c->N * c->K_up);
-    agg_link_kernel<<<(total + 255) / 256, 256, 0, c->stream>>>(c->up.out, total, c->head, c->next, c->uni, c->ctrl,
-                                                                 (u32)c->d);
+    agg_link_kernel<<<(total + 255) / 256, 256, 0, c->stream>>>(c->up.out, total, (u32)c->K_up, c->head, c->next, c->slots,
+                                                                 c->slot_row_words, c->uni, c->ctrl, (u32)c->d);
     TK_LAUNCH_CHECK();
     c->launches += 1;
     return run_server(c, w_dev, alpha, mode);

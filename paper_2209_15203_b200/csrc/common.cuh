@@ -154,6 +154,23 @@ __device__ __forceinline__ float sq4(uint4 v, float acc) {
     return fmaf(a, a, fmaf(b, b, fmaf(c, c, fmaf(e, e, acc))));
 }
 
+// Slot filing of the server step (few workers), given what the compare-and-swap on head[idx] returned: 0 means this entry was the
+// first at the coordinate and owns it (its value stays where it is, in the message); otherwise the
+// word holds the owner's entry number + 1, and this entry marks the coordinate as shared (top bit),
+// sets its worker's bit in the 128-bit mask that opens the owner's row of the slot table and leaves
+// its value in its worker's column of that row.  Nothing here waits for a result.
+constexpr u32 kSharedBit = 0x80000000u;
+constexpr u32 kSlotMaskWords = 4;
+
+__device__ __forceinline__ void file_in_slot(u32* head, u32* slots, u32 row_words, u32 seen, u32 idx, u32 worker,
+                                             u32 bits) {
+    if (seen == 0) return;
+    if (!(seen & kSharedBit)) atomicOr(&head[idx], kSharedBit);
+    u32* row = slots + (size_t)((seen & ~kSharedBit) - 1) * row_words;
+    atomicOr(row + (worker >> 5), 1u << (worker & 31u));
+    row[kSlotMaskWords + worker] = bits;
+}
+
 // Append the lanes with `pred` to a list whose fill counter is *counter.
 // Every lane of the warp must call.  The counter always advances by the number
 // of appending lanes; entries that would land beyond `cap` are dropped (the

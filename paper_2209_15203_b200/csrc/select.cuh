@@ -662,6 +662,11 @@ struct LinkArgs {
     float* zero_src;
     size_t zero_stride;
     int stats;  // diagnostics: add the squares of the emitted values to RowState.sel_sq
+    // Few workers: instead of chains, head[idx] keeps the first entry e0 to arrive at the coordinate;
+    // every later entry sets the word's top bit and files its value in row e0 of the slot table
+    // (row_words words per row, all zero at rest); see aggregate.cuh.
+    u32* slots;
+    u32 row_words;
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
@@ -678,8 +683,14 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
     if (link.zero_src) link.zero_src[(size_t)row * link.zero_stride + idx] = 0.0f;
     if (link.head) {
         u32 e = (link.row_base + row) * (u32)out_stride + slot;
-        if (idx < link.d) link.next[e] = atomicExch(&link.head[idx], e + 1);
-        else { link.next[e] = 0; raise_status(ctrl, -5); }
+        if (idx >= link.d) {
+            link.next[e] = 0;
+            raise_status(ctrl, -5);
+        } else if (link.slots) {
+            file_in_slot(link.head, link.slots, link.row_words, atomicCAS(&link.head[idx], 0u, e + 1), idx, link.row_base + row, bits);
+        } else {
+            link.next[e] = atomicExch(&link.head[idx], e + 1);
+        }
     }
 }
 
@@ -853,8 +864,10 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                 u32 idx = 0xffffffffu - (u32)eck[k];
                 if (slot < Keff && idx < 0x80000000u) {
                     if (apply.w) fetched[k] = __float_as_uint(apply.w[idx]);
-                    if (link.head && idx < link.d)
-                        fetched[k] = atomicExch(&link.head[idx], (link.row_base + row) * (u32)out_stride + slot + 1);
+                    if (link.head && idx < link.d) {
+                        const u32 e1 = (link.row_base + row) * (u32)out_stride + slot + 1;
+                        fetched[k] = link.slots ? atomicCAS(&link.head[idx], 0u, e1) : atomicExch(&link.head[idx], e1);
+                    }
                 }
                 ++slot;
             }
@@ -875,8 +888,9 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                     if (link.zero_src) link.zero_src[(size_t)row * link.zero_stride + idx] = 0.0f;
                     if (link.head) {
                         u32 e = (link.row_base + row) * (u32)out_stride + slot;
-                        if (idx < link.d) link.next[e] = fetched[k];
-                        else { link.next[e] = 0; raise_status(ctrl, -5); }
+                        if (idx >= link.d) { link.next[e] = 0; raise_status(ctrl, -5); }
+                        else if (link.slots) file_in_slot(link.head, link.slots, link.row_words, fetched[k], idx, link.row_base + row, bits);
+                        else link.next[e] = fetched[k];
                     }
                     if (link.stats) sel_sq += (double)__uint_as_float(bits) * (double)__uint_as_float(bits);
                 }
