@@ -76,9 +76,63 @@ u32 candidate_capacity(int64_t d, int64_t K) {
     return (u32)cap;
 }
 
-SelectLayout select_layout(int64_t rows, int64_t d, int64_t K) {
+bool sampled_path(int64_t d, int64_t K, bool force_general) { return !force_general && d >= 131072 && K * 64 <= d; }
+
+// The sample the prediction kernel takes of every row: ~128*d/K values (about 128 members of the top K;
+// fewer when that would take more than the kernel's loads per thread), as whole 128-byte lines.
+struct SamplePlan {
+    int turns;        // 16-byte loads per sampling thread
+    u64 stride_fp;    // 32.32 fixed-point distance between the sampled lines
+    u32 rank;         // the bound is the rank-th largest of the per-thread-pair maxima
+    double crowd;     // see below
+};
+
+// `light`: the two-CTAs-per-SM variant (many rows); `fused`: with error memories, two loads per value.
+// crowd = 8 * rank / sampled fraction.  A thread pair keeps one maximum of 8 neighbouring sampled values,
+// so when the K largest sit packed in one block of R values the sample holds about R*fraction/8 maxima
+// from it; if that is below `rank` the bound drops to the level of the values outside and the whole
+// block qualifies.  Lists of `crowd` entries (plus slack) still hold such a block, and a bigger block
+// fills `rank` maxima by itself.
+SamplePlan plan_sample(int64_t d, int64_t K, bool light, bool fused) {
+    SamplePlan sp;
+    const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
+    int64_t max_turns = light ? kPredictLightTurns : kPredictMaxTurns;
+    if (fused) max_turns /= 2;
+    int64_t want = (128 * (d / K) + per_turn - 1) / per_turn;
+    int64_t lim = d / (8 * per_turn) < max_turns ? d / (8 * per_turn) : max_turns;
+    sp.turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
+    if (sp.turns < 1) sp.turns = 1;
+    u64 lines = (u64)sp.turns * (2 * kSampleSlots / 8);
+    sp.stride_fp = ((u64)(d - 32) << 32) / (lines - 1);                  // run g starts near g*(d-32)/(lines-1)
+    double ks = (double)K * 32.0 * (double)lines / (double)d;          // expected top-K members in the sample
+    double r = ceil(ks + 6.0 * sqrt(ks) + 4.0);
+    sp.rank = (u32)(r > kSampleSlots / 2 ? kSampleSlots / 2 : r);
+    sp.crowd = 8.0 * (double)sp.rank * (double)d / (32.0 * (double)lines);
+    return sp;
+}
+
+constexpr int kSmsAssumed = 148;  // B200; only sizes the lists below (a wrong guess costs speed in a rare case, nothing else)
+
+bool light_sampling(int64_t rows, int sms) { return rows * kPredictCtas > 2 * (int64_t)sms; }
+
+// Candidate capacity per row of the batched selection: room for 4K + 8192 entries and, on the sampled
+// path, for a block of large values the sample under-counts (plan_sample), at most 2^20 entries.
+u32 wide_capacity(int64_t rows, int64_t d, int64_t K) {
+    int64_t cap = candidate_capacity(d, K);
+    if (!sampled_path(d, K, false)) return (u32)cap;
+    bool light = light_sampling(rows, kSmsAssumed);
+    double crowd = plan_sample(d, K, light, false).crowd, crowd_ef = plan_sample(d, K, light, true).crowd;
+    if (crowd_ef > crowd) crowd = crowd_ef;
+    int64_t want = (int64_t)(1.15 * crowd) + 2 * K;
+    if (want > ((int64_t)1 << 20)) want = (int64_t)1 << 20;
+    if (want > cap) cap = want;
+    if (cap > d) cap = d;
+    return (u32)cap;
+}
+
+SelectLayout select_layout(int64_t rows, int64_t d, int64_t K, bool wide = true) {
     SelectLayout L;
-    L.cap = candidate_capacity(d, K);
+    L.cap = wide ? wide_capacity(rows, d, K) : candidate_capacity(d, K);
     int64_t nv = (d + 3) / 4;
     int64_t tf = (nv + kFilterTileVecs - 1) / kFilterTileVecs, tg = (nv + kGeneralTileVecs - 1) / kGeneralTileVecs;
     int64_t te = (nv + kFilterEfTileVecs - 1) / kFilterEfTileVecs;
@@ -373,7 +427,7 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
-    const bool predict = !force_general && d >= 131072 && K * 64 <= d;
+    const bool predict = sampled_path(d, K, force_general);
     bool fused = ef.eps != nullptr && predict && ((((uintptr_t)x) ^ ((uintptr_t)ef.eps)) & 15u) == 0;
     if (ef.eps && !fused) {
         size_t n = (size_t)rows * (size_t)d;
@@ -389,22 +443,12 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
     u64 stride_fp = 0;
     u32 rank = 0;
     if (predict) {
-        // sample ~128*d/K values per row (about 128 members of the top K; fewer when that would take
-        // more than kPredictMaxTurns loads per thread), as whole 128-byte lines
-        const int64_t per_turn = 4 * 2 * (int64_t)kSampleSlots;          // values read per turn
-        int64_t max_turns = fused ? kPredictMaxTurns / 2 : kPredictMaxTurns;
-        // many rows: the sampling CTAs of all rows should fit few waves, so cap the loads per thread
-        // at what the two-CTAs-per-SM variant holds (the sample only sets how many candidates pass)
-        if (rows * kPredictCtas > 2 * (int64_t)di->sms) max_turns = fused ? kPredictLightTurns / 2 : kPredictLightTurns;
-        int64_t want = (128 * (d / K) + per_turn - 1) / per_turn;
-        int64_t lim = d / (8 * per_turn) < max_turns ? d / (8 * per_turn) : max_turns;
-        turns = (int)(want < 1 ? 1 : (want > lim ? lim : want));
-        if (turns < 1) turns = 1;
-        u64 lines = (u64)turns * (2 * kSampleSlots / 8);
-        stride_fp = ((u64)(d - 32) << 32) / (lines - 1);                  // run g starts near g*(d-32)/(lines-1)
-        double ks = (double)K * 32.0 * (double)lines / (double)d;          // expected top-K members in the sample
-        double r = ceil(ks + 6.0 * sqrt(ks) + 4.0);
-        rank = (u32)(r > kSampleSlots / 2 ? kSampleSlots / 2 : r);
+        // many rows: the sampling CTAs of all rows should fit few waves, so cap the loads per thread at
+        // what the two-CTAs-per-SM variant holds (the sample only sets how many candidates pass)
+        SamplePlan sp = plan_sample(d, K, light_sampling(rows, di->sms), fused);
+        turns = sp.turns;
+        stride_fp = sp.stride_fp;
+        rank = sp.rank;
     }
     for (int64_t r0 = 0; r0 < rows; r0 += kMaxRowsPerLaunch) {
         int nr = (int)(rows - r0 < kMaxRowsPerLaunch ? rows - r0 : kMaxRowsPerLaunch);
@@ -420,13 +464,13 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             const bool light = turns <= (fused ? kPredictLightTurns / 2 : kPredictLightTurns);
             dim3 pg(kPredictCtas, nr);
             if (fused && light)
-                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb);
             else if (fused)
-                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb);
             else if (light)
-                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb);
             else
-                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, rs, smax, ar, efb);
+                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             u32 tprf = fused ? b.tpr_filter_ef : b.tpr_filter;
@@ -1197,7 +1241,7 @@ int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int3
     // size check first, in 64-bit arithmetic that cannot wrap for any accepted rows/d/K
     if ((double)rows * ((double)candidate_capacity(d, K) + 2.0 * (double)K) * 8.0 > (double)TK_NOALLOC_SCRATCH_BYTES)
         return TK_ERR_TOO_LARGE;
-    SelectLayout SL = select_layout(rows, d, K);
+    SelectLayout SL = select_layout(rows, d, K, false);
     SortLayout QL = sort_layout(rows, K);
     size_t off_ctrl = SL.bytes + QL.bytes;
     if (off_ctrl + align_up(sizeof(Ctrl)) > (size_t)TK_NOALLOC_SCRATCH_BYTES) return TK_ERR_TOO_LARGE;

@@ -55,7 +55,7 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
 // fit an SM (used when the rows are many and the sample per row is small).
 template <bool kEF, bool kLight>
 __global__ void __launch_bounds__(kPredictThreads, kLight ? 2 : 1)
-predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank,
+predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank, u32 K,
                RowState* rs, u32* smax, RowState* also_reset, EfArgs ef) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ u32 sh_scratch[33];
@@ -143,7 +143,13 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
         prefix |= b << shift;
         need -= above;
     }
-    if (threadIdx.x == 0) reset_state(rs + row, (u64)prefix << 32, 0u);
+    // A bound of key 0 means the row is nearly all zeros.  Taking every component would overflow the
+    // list; (key 0, index K-1) is a valid bound as well: it admits every non-zero and the zeros among
+    // the first K components, and if fewer than K components are non-zero, the first K components
+    // hold enough zeros to make up the difference (zeros rank by ascending index).
+    u64 lo = (u64)prefix << 32;
+    if (prefix == 0) lo = composite(0u, K - 1u);
+    if (threadIdx.x == 0) reset_state(rs + row, lo, 0u);
 }
 
 // eps <- eps + alpha * g over n values (the compensated vector, for the paths that do not
@@ -331,18 +337,26 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, 
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) sq = sq4(v[u], sq);
     }
+    if (tk != 0) {
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        bool hit = inb[u] && may_hit(v[u], thr);
-        if (__any_sync(0xffffffffu, hit)) {
-            u32 i0 = g.head + 4u * (j0 + u * THREADS);
-            if (tk == 0) {  // everything in the row qualifies; only the padding lanes must stay out
+        for (int u = 0; u < UNROLL; ++u) {
+            bool hit = inb[u] && may_hit(v[u], thr);
+            // padding lanes hold zeros, whose key is below tk
+            if (__any_sync(0xffffffffu, hit)) consider4(v[u], g.head + 4u * (j0 + u * THREADS), tk, lo, st, rs, cand, cap);
+        }
+    } else {
+        // key 0 in the bound (a row of nearly all zeros, or one where everything qualifies): every
+        // non-zero passes, and the zeros up to the bound's index; exact test per component
+        const u32 last_zero = 0xffffffffu - (u32)lo;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const u32 i0 = g.head + 4u * (j0 + u * THREADS);
+            bool hit = inb[u] && ((((v[u].x | v[u].y | v[u].z | v[u].w) & 0x7fffffffu) != 0u) || i0 <= last_zero);
+            if (__any_sync(0xffffffffu, hit)) {
                 consider(hit, i0 + 0, v[u].x, lo, st, rs, cand, cap);
                 consider(hit, i0 + 1, v[u].y, lo, st, rs, cand, cap);
                 consider(hit, i0 + 2, v[u].z, lo, st, rs, cand, cap);
                 consider(hit, i0 + 3, v[u].w, lo, st, rs, cand, cap);
-            } else {        // padding lanes hold zeros, whose key is below tk
-                consider4(v[u], i0, tk, lo, st, rs, cand, cap);
             }
         }
     }

@@ -121,6 +121,27 @@ def test_rows_whose_prediction_must_fail():
     run_both(x, K)
 
 
+def test_rows_the_sample_misjudges_stay_on_the_single_pass_path():
+    # (a) fewer non-zeros than K: the K-th largest is a zero, zeros rank by index;
+    # (b) the K largest packed into one short block of huge values, which the sample under-counts;
+    # (c) a few more non-zeros than K.  All exact, and none needs the multi-pass path.
+    d, K, rows = 4_000_003, 2_000, 4
+    rng = np.random.default_rng(515)
+    x = np.zeros((rows, d), dtype=np.float32)
+    x[0, rng.choice(d, 700, replace=False)] = rng.standard_normal(700).astype(np.float32)
+    x[0, rng.choice(d, 5000, replace=False)] *= np.float32(-1.0)        # some of the zeros become -0
+    x[1] = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    x[1, 1_234_567:1_234_567 + 20_000] *= np.float32(1000.0)
+    x[2, rng.choice(d, 2_300, replace=False)] = rng.standard_normal(2_300).astype(np.float32)
+    x[3] = (rng.standard_normal(d) * 1e-3).astype(np.float32)
+    ctx = binding.Context(d, rows, K, K, torch.full((rows,), 1.0 / rows))
+    run_both(x, K, ctx=ctx)
+    st = ctx.tk_status()
+    assert st.rows_general == 0, "every row should verify with its sampled bound"
+    assert st.cand_max < 40_000
+    ctx.close()
+
+
 def test_predicted_and_general_paths_agree_bitwise():
     wl = W.workload(2, d=1_170_000, N=6)
     G = W.make_grads(wl, 1, DEV)
