@@ -13,7 +13,7 @@ DEV = "cuda:0"
 EF = binding.TK_MODE_EF
 
 
-def run_ef(wl, steps, mode, K_down=None, force_general=False, misalign=0, alpha=None):
+def run_ef(wl, steps, mode, K_down=None, force_general=False, misalign=0, alpha=None, keep=None):
     K_down = K_down or wl.K_down[0]
     alpha = wl.alpha if alpha is None else alpha
     p = W.make_p(wl)
@@ -31,6 +31,10 @@ def run_ef(wl, steps, mode, K_down=None, force_general=False, misalign=0, alpha=
     G = buf[misalign:misalign + wl.N * wl.d].view(wl.N, wl.d)
     for s in range(steps):
         W.make_grads(wl, s, DEV, out=G, scale=scale)
+        if keep is not None:   # sparse gradients: all but a fraction `keep` of the components are exactly zero
+            gen = torch.Generator(device=DEV)
+            gen.manual_seed(77 + s)
+            G.mul_((torch.rand(G.shape, generator=gen, device=DEV) < keep).to(torch.float32))
         ctx.tk_step(w_dev, G, alpha, mode | EF)
         ref = oracle.ref_step_ef(w, eps, delta, G.cpu().numpy(), wl.K_up, K_down, p.numpy(), alpha, mode)
         what = "config%d ef mode=%d step=%d" % (wl.cid, mode, s)
@@ -81,6 +85,12 @@ def test_short_rows_multi_pass_path(mode):
 def test_ragged_rows_and_unaligned_gradients():
     run_ef(W.workload(5, d=1_000_003, N=3), 3, 1)                  # d % 4 != 0
     run_ef(W.workload(2, d=600_000, N=3), 3, 1, misalign=1)        # gradients not aligned like the memories
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_sparse_gradients_fewer_nonzeros_than_k(mode):
+    # the compensated vectors and the server memory are nearly all zeros: the K-th largest is a zero
+    run_ef(W.workload(2, d=1_170_004, N=4), 4, mode, keep=2e-4)
 
 
 def test_forced_multi_pass_path():

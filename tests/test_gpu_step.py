@@ -182,6 +182,23 @@ def test_workers_that_agree(N, noise):
         ctx.close()
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_sparse_gradients_fewer_nonzeros_than_k(mode):
+    # rows of nearly all zeros (some of them -0): the messages are padded with the first zeros by index
+    wl = W.workload(2, d=1_170_004, N=5)
+    ctx = make_ctx(wl, wl.K_down[0])
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(4242)
+    w_dev = W.make_w(wl, DEV)
+    w_ref = w_dev.cpu().numpy()
+    for s in range(2):
+        G = W.make_grads(wl, s, DEV)
+        G.mul_((torch.rand(G.shape, generator=gen, device=DEV) < 3e-4).to(torch.float32))
+        w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, mode, wl.K_down[0], "sparse rows mode=%d step=%d" % (mode, s))
+        assert ctx.tk_status().rows_general == 0
+    ctx.close()
+
+
 def test_step_host_matches_device_step():
     wl = W.workload(2, d=500_000, N=4)
     G = W.make_grads(wl, 0, DEV)
