@@ -32,11 +32,11 @@
 
 namespace tk {
 
-// Threads every entry of a gathered message buffer onto its coordinate's chain — what the
-// uplink selection's emission does on the fly when the messages are produced on this GPU.
-// Also resets the union's state for the step.
-constexpr int kSlotWorkers = 128;  // the slot table is used up to this many workers
+constexpr int kSlotWorkers = 128;  // the slot table is used up to this many workers (its mask has 128 bits)
 
+// Files every entry of a gathered message buffer under its coordinate — what the uplink
+// selection's emission does on the fly when the messages are produced on this GPU.
+// Also resets the union's state for the step.
 __global__ void __launch_bounds__(256)
 agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u32* next, u32* slots, u32 row_words,
                 RowState* uni, Ctrl* ctrl, u32 d) {
@@ -63,7 +63,7 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
                   u32* head, const u32* __restrict__ next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
                   int stats) {
-    dependency_wait();   // the chains are built by the kernel before
+    dependency_wait();   // the entries are filed by the kernel before
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
     u32 j = 0, own_bits = 0;
