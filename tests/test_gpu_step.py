@@ -199,6 +199,37 @@ def test_sparse_gradients_fewer_nonzeros_than_k(mode):
     ctx.close()
 
 
+def test_random_problems_sweep():
+    # many shapes at every alignment: short rows (multi-pass path) and rows long enough for the sampled
+    # path; N from 1 to 140 (slot table up to 128 workers, chains above); coarse values make the workers
+    # share coordinates and tie; K_down below and above the union size
+    rng = np.random.default_rng(220915)
+    for case in range(24):
+        long_rows = case % 4 == 3
+        N = int(rng.integers(1, 9)) if long_rows else int(rng.choice([1, 2, 3, 5, 17, 64, 129, 140]))
+        d = int(rng.integers(140_000, 400_000)) if long_rows else int(rng.integers(4, 9_000))
+        K_up = int(rng.integers(1, max(2, d // (200 if long_rows else 12))))
+        K_down = int(rng.integers(1, min(d, 2 * N * K_up) + 1))
+        p = torch.from_numpy(rng.dirichlet(np.ones(N)).astype(np.float32))
+        wl = W.workload(1, d=d, N=N)
+        wl = wl.__class__(**{**wl.__dict__, "K_up": K_up, "K_down": (K_down,)})
+        for mode in (0, 1):
+            ctx = binding.Context(d, N, K_up, K_down, p)
+            _P[id(ctx)] = p.numpy()
+            w_dev = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+            w_ref = w_dev.cpu().numpy()
+            for s in range(2):
+                Gh = rng.standard_t(3, (N, d)) * 1e-2
+                if case % 3 == 0:
+                    Gh = np.round(Gh * 32) / 32
+                if case % 5 == 0 and N > 1:
+                    Gh[1:] = Gh[0] * (1 + 0.05 * rng.standard_normal((N - 1, d)))
+                G = torch.from_numpy(Gh.astype(np.float32)).to(DEV)
+                w_ref = check_step(ctx, wl, w_dev, w_ref, G, 0.3, mode, K_down,
+                                   "sweep case %d N=%d d=%d K=%d/%d mode=%d step=%d" % (case, N, d, K_up, K_down, mode, s))
+            ctx.close()
+
+
 def test_step_host_matches_device_step():
     wl = W.workload(2, d=500_000, N=4)
     G = W.make_grads(wl, 0, DEV)
