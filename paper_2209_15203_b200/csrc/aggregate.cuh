@@ -43,7 +43,7 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u3
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) {
         uni->lo = 0; uni->cand_count = 0; uni->max_key = 0; uni->out_count = 0; uni->flags = 0;
-        uni->sum_sq = 0.0; uni->sel_sq = 0.0; uni->nnz = 0;
+        uni->sum_sq = 0.0; uni->sel_sq = 0.0; uni->nnz = 0; uni->min_key = 0xffffffffu;
     }
     if (e >= total) return;
     u32 j = up[e].x;
@@ -167,17 +167,20 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     // append (j, g_j) to the union list: one counter update and one maximum per CTA (every entry
     // of every worker passes through here; per-warp atomics on the two words would serialise)
     __shared__ u32 sh_scratch[33];
-    __shared__ u32 sh_base, sh_max;
-    if (threadIdx.x == 0) sh_max = 0;
+    __shared__ u32 sh_base, sh_max, sh_min;
+    if (threadIdx.x == 0) { sh_max = 0; sh_min = 0xffffffffu; }
     u32 bits = __float_as_uint(acc);
     u32 owners;
     u32 incl = block_inclusive_scan(owner ? 1u : 0u, sh_scratch, &owners);
     u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
     if (lane_id() == 0 && wm) atomicMax(&sh_max, wm);
+    u32 wn = __reduce_min_sync(0xffffffffu, owner ? key_of(bits) : 0xffffffffu);
+    if (lane_id() == 0 && wn != 0xffffffffu) atomicMin(&sh_min, wn);
     __syncthreads();
     if (threadIdx.x == 0 && owners) {
         sh_base = atomicAdd(&uni->cand_count, owners);
         atomicMax(&uni->max_key, sh_max);  // the downlink selection wants the largest aggregated magnitude
+        atomicMin(&uni->min_key, sh_min);  // ... and the smallest
     }
     __syncthreads();
     if (owner) {

@@ -238,7 +238,7 @@ struct tk_ctx {
     u32 slot_row_words = 0;
     uint2* U = nullptr;        // [ucap] aggregate over the union
     uint2* sel = nullptr;      // [ucap] downlink message (unordered)
-    u32* ghist = nullptr;      // [3][kHistBins] histograms of the grid-wide select, zero at rest
+    u32* ghist = nullptr;      // [kGridScratchWords] scratch of the grid-wide select, zero at rest
     u32 ucap = 0;
     // host state
     int force_general = 0;
@@ -329,7 +329,7 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
     L.off_slots = o;  o += align_up(L.slot_words * sizeof(u32));
     L.off_U = o;      o += align_up((size_t)ucap * sizeof(uint2));
     L.off_sel = o;    o += align_up((size_t)ucap * sizeof(uint2));
-    L.off_ghist = o;  o += align_up((size_t)3 * kHistBins * sizeof(u32));
+    L.off_ghist = o;  o += align_up((size_t)kGridScratchWords * sizeof(u32));
     L.bytes = o;
     return L;
 }
@@ -659,7 +659,7 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
               cudaMemsetAsync(c->up.rs, 0, (size_t)N * sizeof(RowState), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->up.hist, 0, (size_t)N * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->uni, 0, sizeof(RowState), c->stream) == cudaSuccess &&
-              cudaMemsetAsync(c->ghist, 0, (size_t)3 * kHistBins * sizeof(u32), c->stream) == cudaSuccess &&
+              cudaMemsetAsync(c->ghist, 0, (size_t)kGridScratchWords * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->head, 0, (size_t)d * sizeof(u32), c->stream) == cudaSuccess &&
               (!c->slots || cudaMemsetAsync(c->slots, 0, L.slot_words * sizeof(u32), c->stream) == cudaSuccess) &&
               cudaMemcpyAsync(c->p, p_host, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream) ==

@@ -62,6 +62,10 @@ constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 #define TK_SELECT_PER_THREAD 8
 #endif
 constexpr int kSelectPerThread = TK_SELECT_PER_THREAD;  // candidates per thread the cluster size aims at
+constexpr int kRankMax = 256;          // a bucket of at most this many candidates is ranked directly (cnt^2 compares) instead of refined
+// Global scratch of the grid-wide select: three histograms, a counter (4 words) and a list of kRankMax
+// composite keys; all but the list must be zero when the kernel starts, and are when it ends.
+constexpr int kGridScratchWords = 3 * kHistBins + 4 + 2 * kRankMax;
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path
 constexpr u32 kRowNoFilter = 2u;       // RowState.flags: no filter pass has read this row
@@ -82,7 +86,7 @@ struct RowState {
     double sum_sq;   // sum of squares of the whole vector
     double sel_sq;   // sum of squares of the emitted entries
     u32 nnz;         // union list: entries whose value is not zero
-    u32 pad;
+    u32 min_key;     // union list: smallest key among its entries (lower end of the downlink selection's first range)
 };
 
 // Step-wide control block.

@@ -49,6 +49,7 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->sum_sq = 0.0;
     r->sel_sq = 0.0;
     r->nnz = 0;
+    r->min_key = 0xffffffffu;
 }
 
 // kLight: at most kPredictLightTurns loads per thread; needs half the registers, so two CTAs
@@ -726,8 +727,12 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     __shared__ u32 sh_tot[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
+    __shared__ u64 sh_list[kRankMax];  // the bucket that gets ranked directly (cluster: gathered in CTA 0's copy)
+    __shared__ u32 sh_list_n;
+    __shared__ u64 sh_T;
     cg::cluster_group cluster = cg::this_cluster();
     cg::grid_group grid = cg::this_grid();
+    if (threadIdx.x == 0) sh_list_n = 0;  // read by peers only after a cluster barrier
     dependency_wait();   // candidates and bounds come from the kernels before
     allow_dependents();
     const u32 CS = kGrid ? gridDim.x : cluster.num_blocks();
@@ -762,10 +767,11 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     u64 T = 1;  // emit entries with ck >= T (absent ones are 0)
     if (C > Keff) {
         u64 lo = max(r->lo, 1ull);
+        if (kGrid) lo = max(lo, (u64)r->min_key << 32);  // the union list knows its smallest key (never above its largest)
         u64 hi = ((u64)r->max_key << 32) | 0xffffffffull;
         if (hi < lo) hi = lo;
         u32 need = Keff;
-        bool found = false;
+        bool found = false, ranked = false;
         for (int level = 0; level < 8 && !found; ++level) {
             u32* hist = sh_hist[level & 1];
             u64 width = hi - lo;
@@ -820,10 +826,59 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             u64 blo = lo + ((u64)b << s);
             u64 bhi = blo + ((1ull << s) - 1ull);
             if (bhi > hi) bhi = hi;
-            if (need == sh_tot[b]) { T = blo; found = true; }
+            const u32 cnt = sh_tot[b];
             lo = blo;
             hi = bhi;
             __syncthreads();
+            if (need == cnt) {
+                T = blo;
+                found = true;
+            } else if (cnt <= (u32)kRankMax) {
+                // Few entries left in the bucket: gather them in one place, let every CTA copy them and
+                // find the need-th largest by counting, for each entry, the entries above it (composite
+                // keys are all different, so exactly one entry has need-1 above it).  One barrier instead
+                // of one or two more levels.
+                u64* gather = kGrid ? (CS == 1 ? sh_list : reinterpret_cast<u64*>(ghist + 3 * kHistBins + 4))
+                                  : cluster.map_shared_rank(sh_list, 0);
+                u32* fill = kGrid ? (CS == 1 ? &sh_list_n : ghist + 3 * kHistBins)
+                                  : cluster.map_shared_rank(&sh_list_n, 0);
+                const u64 width2 = hi - lo;
+#pragma unroll
+                for (int k = 0; k < kSelectRegs; ++k) {
+                    if ((u32)k >= nslots) break;
+                    if (eck[k] - lo <= width2) gather[atomicAdd(fill, 1u)] = eck[k];
+                }
+                for (u32 i = rest; i < C; i += stride) {
+                    uint2 e = list[i];
+                    u64 ck = composite(key_of(e.y), e.x);
+                    if (ck - lo <= width2) gather[atomicAdd(fill, 1u)] = ck;
+                }
+                if (kGrid && CS == 1) {
+                    __syncthreads();
+                } else if (kGrid) {
+                    grid.sync();  // the list is complete; nobody reads the histograms or the counter any more
+                    if (rank == 0) {
+                        for (int i = threadIdx.x; i < 3 * kHistBins + 4; i += kSelectThreads) ghist[i] = 0;
+                    }
+                    for (u32 i = threadIdx.x; i < cnt; i += kSelectThreads) sh_list[i] = __ldcg(gather + i);
+                    __syncthreads();
+                } else {
+                    cluster.sync();
+                    if (rank != 0)
+                        for (u32 i = threadIdx.x; i < cnt; i += kSelectThreads) sh_list[i] = gather[i];
+                    __syncthreads();
+                }
+                for (u32 i = threadIdx.x; i < cnt; i += kSelectThreads) {
+                    const u64 me = sh_list[i];
+                    u32 above = 0;
+                    for (u32 o = 0; o < cnt; ++o) above += sh_list[o] > me ? 1u : 0u;
+                    if (above == need - 1) sh_T = me;
+                }
+                __syncthreads();
+                T = sh_T;
+                found = true;
+                ranked = true;
+            }
         }
         if (!found) {
             T = lo;
@@ -832,10 +887,13 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         if (kGrid && CS == 1) {
             // nothing was exchanged
         } else if (kGrid) {
-            // leave ghist all zero for the next launch: once everybody has read the last level
-            grid.sync();
-            if (rank == 0)
-                for (int b = threadIdx.x; b < 3 * kHistBins; b += kSelectThreads) ghist[b] = 0;
+            // leave the scratch all zero for the next launch: once everybody has read the last level
+            // (the ranking step has done both already)
+            if (!ranked) {
+                grid.sync();
+                if (rank == 0)
+                    for (int b = threadIdx.x; b < 3 * kHistBins; b += kSelectThreads) ghist[b] = 0;
+            }
         } else {
             cluster.sync();  // no CTA leaves while a peer may still read its histograms
         }
