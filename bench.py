@@ -170,8 +170,9 @@ def main():
                     "sampled single-pass one")
     ap.add_argument("--no-graph", action="store_true", help="issue every step as plain stream launches instead of "
                     "replaying captured CUDA graphs (tk_set_graph)")
-    ap.add_argument("--profile-every", type=int, default=4, help="timestamp the streaming kernel of every n-th timed "
-                    "step (such a step is issued as plain launches)")
+    ap.add_argument("--profile-every", type=int, default=0, help="timestamp the streaming kernel of every n-th timed "
+                    "step (such a step is issued as plain launches, which costs it some tens of microseconds); "
+                    "default: about eight samples over the run, at most every 10th step")
     ap.add_argument("--agree", type=float, default=None, metavar="C",
                     help="workers see noisy copies of one shared vector, row_q = base * (1 + C z_q), instead of "
                          "independent rows: their selections then mostly coincide (union near K)")
@@ -179,6 +180,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.profile_every <= 0:
+        args.profile_every = max(1, min(10, args.steps // 8))
 
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
