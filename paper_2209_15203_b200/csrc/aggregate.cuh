@@ -69,8 +69,10 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     u32 j = 0, own_bits = 0;
     float acc = 0.0f;
     bool shared = false;
+    float own_p = 0.0f;
     if (e < total) {
         uint2 mine = up[e];
+        own_p = p[e / K_up];  // asked for now, not after the coordinate's word has come back
         j = mine.x;
         own_bits = mine.y;
         u32 h = j < d ? __ldcg(&head[j]) : 0u;
@@ -81,7 +83,7 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     if (owner && slots) {
         const u32 own_q = e / K_up;
         if (!shared) {
-            acc = __fadd_rn(acc, __fmul_rn(p[own_q], __uint_as_float(own_bits)));
+            acc = __fadd_rn(acc, __fmul_rn(own_p, __uint_as_float(own_bits)));
         } else {
             u32* row = slots + (size_t)e * row_words;
             const uint4 m = __ldcg(reinterpret_cast<const uint4*>(row));
