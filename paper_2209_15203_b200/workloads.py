@@ -32,7 +32,7 @@ def k_from_ratio(d: int, num: int, den: int) -> int:
 
 @dataclass(frozen=True)
 class Workload:
-    cid: int                      # configuration number (1..5 benchmark workloads, 6..9 paper shapes)
+    cid: int                      # configuration number (1..5 benchmark workloads, 6..10 paper shapes)
     name: str
     N: int                        # workers (rows)
     d: int                        # vector length
@@ -90,6 +90,10 @@ def _cfg(cid: int, d: Optional[int] = None) -> Workload:
         d = d or 29_034
         K = k_from_ratio(d, 1, 1000)
         return Workload(9, "paper-fmnist-cnn", 20, d, K, (K,), 10, (0, 1), "student", 6, 1e-4, 1e-2, "uniform")
+    if cid == 10:  # MLP [784,64,10] on MNIST, 100 workers
+        d = d or 50_890
+        K = k_from_ratio(d, 1, 1000)
+        return Workload(10, "paper-mnist-mlp", 100, d, K, (K,), 10, (0, 1), "gauss", 4, 1e-4, 1e-2, "uniform")
     raise ValueError("unknown configuration %r" % cid)
 
 

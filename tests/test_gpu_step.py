@@ -90,7 +90,7 @@ def test_scaled_configs_every_step(cid, d):
     run_workload(wl, 3)
 
 
-@pytest.mark.parametrize("cid", [6, 8, 9])
+@pytest.mark.parametrize("cid", [6, 8, 9, 10])
 def test_paper_shaped_workloads(cid):
     # N = 20..100 workers, d not a multiple of 4 (rows start at every alignment), tiny K
     wl = W.workload(cid)

@@ -17,8 +17,8 @@ def test_k_values_of_the_five_configurations():
 
 
 def test_paper_shapes():
-    assert [(W.workload(c).N, W.workload(c).d, W.workload(c).K_up) for c in (6, 7, 8, 9)] == \
-        [(100, 242_762, 243), (20, 20_040_522, 20_041), (50, 1_199_882, 1_200), (20, 29_034, 30)]
+    assert [(W.workload(c).N, W.workload(c).d, W.workload(c).K_up) for c in (6, 7, 8, 9, 10)] == \
+        [(100, 242_762, 243), (20, 20_040_522, 20_041), (50, 1_199_882, 1_200), (20, 29_034, 30), (100, 50_890, 51)]
 
 
 def test_block_layout_covers_d():
