@@ -42,7 +42,7 @@ int device_info(DeviceInfo** out) {
             per_sm < 1)
             return TK_ERR_CUDA;
         di.general_grid = per_sm * di.sms;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel<true>, kSelectThreads, 0) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel<true, false>, kSelectThreads, 0) != cudaSuccess ||
             per_sm < 1)
             return TK_ERR_CUDA;
         di.select_grid = per_sm * di.sms;
@@ -395,8 +395,31 @@ int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
 int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, size_t list_stride, u32 cap,
                   RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
     u32* no_ghist = nullptr;
-    return launch_dependent(select_kernel<false>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, lists,
-                            list_stride, cap, rs, K, out, out_stride, apply, link, ctrl, no_ghist);
+    DenseArgs no_dense = {nullptr, nullptr, 0};
+    return launch_dependent(select_kernel<false, false>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, lists,
+                            list_stride, cap, rs, K, out, out_stride, apply, link, ctrl, no_ghist, no_dense);
+}
+
+// CTAs per row when the selection reads short rows directly: enough to keep (nearly) the whole row in
+// registers (what does not fit is read again at every level).  0 when the row is too long for that or the
+// clusters of all rows would not fit one wave — measured: 100 rows of 51k as 400 CTAs take longer than
+// the multi-pass kernel, 20 rows of 29k as 80 CTAs take half as long.
+int dense_cluster_size(int64_t d, int64_t rows, int sms) {
+    const int64_t held = (int64_t)kSelectRegs * kSelectThreads;  // entries one CTA keeps in registers
+    int cs = 1;
+    while (cs < 8 && cs * held < d) cs *= 2;
+    if (cs * held * 9 / 8 < d || rows * cs > (int64_t)sms) return 0;  // a remainder of an eighth may be re-read
+    return cs;
+}
+
+// The same selection straight from short rows (no candidate lists, no bound).
+int launch_select_dense(cudaStream_t stream, int rows, int cs, const float* x, int64_t d, RowState* rs, u32 K, uint2* out,
+                        ApplyArgs apply, LinkArgs link, Ctrl* ctrl, RowState* also_reset, bool stats) {
+    u32* no_ghist = nullptr;
+    const uint2* no_lists = nullptr;
+    DenseArgs dense = {x, also_reset, stats ? 1 : 0};
+    return launch_dependent(select_kernel<false, true>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, no_lists,
+                            (size_t)d, (u32)d, rs, K, out, (size_t)K, apply, link, ctrl, no_ghist, dense);
 }
 
 // One long list selected by the whole grid (cooperative launch).
@@ -404,9 +427,10 @@ int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap
                        ApplyArgs apply, Ctrl* ctrl, u32* ghist, bool stats) {
     size_t stride = cap;
     LinkArgs nolink = {nullptr, nullptr, 0, 0, nullptr, 0, stats ? 1 : 0};
+    DenseArgs no_dense = {nullptr, nullptr, 0};
     void* args[] = {(void*)&list, (void*)&stride, (void*)&cap, (void*)&rs,  (void*)&K,    (void*)&out,
-                    (void*)&stride, (void*)&apply, (void*)&nolink, (void*)&ctrl, (void*)&ghist};
-    if (cudaLaunchCooperativeKernel((void*)select_kernel<true>, dim3(ctas), dim3(kSelectThreads), args, 0, stream) !=
+                    (void*)&stride, (void*)&apply, (void*)&nolink, (void*)&ctrl, (void*)&ghist, (void*)&no_dense};
+    if (cudaLaunchCooperativeKernel((void*)select_kernel<true, false>, dim3(ctas), dim3(kSelectThreads), args, 0, stream) !=
         cudaSuccess) {
         cudaGetLastError();
         return TK_ERR_CUDA;
@@ -439,6 +463,9 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
         x = ef.eps;            // from here on this is an ordinary selection over eps
         ef.eps = nullptr;
     }
+    // rows too short for a sampled bound are selected from directly (unless the multi-pass path is forced)
+    const int dense_cs = (!predict && !force_general) ? dense_cluster_size(d, rows < kMaxRowsPerLaunch ? rows : kMaxRowsPerLaunch, di->sms) : 0;
+    const bool dense = dense_cs > 0;
     int turns = 1;
     u64 stride_fp = 0;
     u32 rank = 0;
@@ -501,6 +528,19 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             if (fused) xb = efb.eps;  // the compensated vector now sits in eps: what a re-filter must read
             if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 2;
+        } else if (dense) {
+            // short rows: one kernel selects straight from the rows
+            LinkArgs lk = link;
+            lk.row_base = (u32)r0;
+            lk.stats = stats ? 1 : 0;
+            if (lk.zero_src) lk.zero_src += (size_t)r0 * lk.zero_stride;
+            if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
+            rc = launch_select_dense(stream, nr, dense_cs, xb, d, rs, (u32)K, out, apply, lk, ctrl,
+                                     r0 == 0 ? also_reset : nullptr, stats);
+            if (rc != TK_OK) return rc;
+            if (ev1 && r0 == 0) cudaEventRecord(ev1, stream);
+            *launches += 1;
+            continue;
         } else {
             reset_rows_kernel<<<(nr + 255) / 256, 256, 0, stream>>>(rs, nr, r0 == 0 ? also_reset : nullptr);
             TK_LAUNCH_CHECK();

@@ -15,7 +15,9 @@
 //   select_kernel    one thread-block cluster per row (or, for one long list, the
 //                    whole grid): range-adaptive radix select of the K largest
 //                    composite keys among the candidates, then emission of
-//                    exactly K entries
+//                    exactly K entries.  Few short rows skip the three kernels
+//                    above: the same kernel takes every component of the row
+//                    as a candidate.
 //
 // The result is always the exact Top_K; the sample only decides how many
 // passes over the data it takes.
@@ -686,6 +688,14 @@ struct LinkArgs {
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
 
+// Short rows with no sampled bound: the selection reads the row itself instead of a candidate
+// list (entry i is component i), which replaces the multi-pass kernel and its launches.
+struct DenseArgs {
+    const float* x;          // [rows][list_stride] the rows themselves
+    RowState* also_reset;    // union state to reset for the step (may be NULL)
+    int stats;               // diagnostics: also sum the squares of every row into RowState.sum_sq
+};
+
 __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx, u32 bits, uint2* orow,
                                            size_t out_stride, const ApplyArgs& apply, const LinkArgs& link,
                                            Ctrl* ctrl) {
@@ -719,10 +729,15 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
 //                   lists too long for one cluster (the union of N uplink messages);
 //                   histograms are combined in `ghist` (3 x kHistBins words of global
 //                   memory, all zero when the kernel starts), grid barriers between levels
-template <bool kGrid>
+//
+// kDense (cluster variant only): the "list" of row r is the row dense.x[r][0..cap) itself, every
+// component a candidate; the kernel then also does what the sampling / reset kernels do for
+// the other paths (row state, union state).
+template <bool kGrid, bool kDense = false>
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
-              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl, u32* ghist) {
+              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl, u32* ghist,
+              DenseArgs dense) {
     __shared__ u32 sh_hist[2][kHistBins];  // double-buffered: peers may still read level L while L+1 fills
     __shared__ u32 sh_tot[kHistBins];
     __shared__ u32 sh_scratch[33];
@@ -739,9 +754,24 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     const u32 rank = kGrid ? blockIdx.x : cluster.block_rank();
     const u32 row = kGrid ? 0u : blockIdx.x / CS;
     RowState* r = rs + row;
-    const u32 C = min(r->cand_count, cap);
+    if (kDense) {
+        if (rank == 0 && threadIdx.x == 0) {
+            reset_state(r, 1ull, 0u);
+            r->cand_count = cap;
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            if (dense.also_reset) reset_state(dense.also_reset, 0ull, 0u);
+            ctrl->rows_general = 0;
+        }
+        cluster.sync();  // the row's counters are reset before any CTA of the row adds to them
+    }
+    const u32 C = kDense ? cap : min(r->cand_count, cap);
     const u32 Keff = min(K, C);
-    const uint2* list = lists + (size_t)row * list_stride;
+    const uint2* list = kDense ? nullptr : lists + (size_t)row * list_stride;
+    const float* xrow = kDense ? dense.x + (size_t)row * list_stride : nullptr;
+    auto read_entry = [&](u32 i) -> uint2 {
+        return kDense ? make_uint2(i, __float_as_uint(__ldg(xrow + i))) : list[i];
+    };
     const u32 first = rank * kSelectThreads + threadIdx.x;
     const u32 stride = CS * kSelectThreads;
     const u32 rest = first + kSelectRegs * stride;  // entries from here on are re-read every level
@@ -758,17 +788,31 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         u32 i = first + (u32)k * stride;
         eck[k] = 0;
         if ((u32)k < nslots && i < C) {
-            uint2 e = list[i];
+            uint2 e = read_entry(i);
             eck[k] = composite(key_of(e.y), e.x);
             esign |= (e.y >> 31) << k;
         }
+    }
+    if (kDense && dense.stats) {  // diagnostics: the row's squared norm (no streaming pass reads these rows)
+        float sq = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kSelectRegs; ++k) {
+            if ((u32)k >= nslots) break;
+            float v = __uint_as_float((u32)(eck[k] >> 32));
+            sq = fmaf(v, v, sq);
+        }
+        for (u32 i = rest; i < C; i += stride) {
+            float v = __ldg(xrow + i);
+            sq = fmaf(v, v, sq);
+        }
+        warp_add_double(&r->sum_sq, (double)sq);
     }
 
     u64 T = 1;  // emit entries with ck >= T (absent ones are 0)
     if (C > Keff) {
         u64 lo = max(r->lo, 1ull);
         if (kGrid) lo = max(lo, (u64)r->min_key << 32);  // the union list knows its smallest key (never above its largest)
-        u64 hi = ((u64)r->max_key << 32) | 0xffffffffull;
+        u64 hi = kDense ? 0x7fffffffffffffffull : ((u64)r->max_key << 32) | 0xffffffffull;  // dense: no maximum is known
         if (hi < lo) hi = lo;
         u32 need = Keff;
         bool found = false, ranked = false;
@@ -787,7 +831,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                 if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
             for (u32 i = rest; i < C; i += stride) {
-                uint2 e = list[i];
+                uint2 e = read_entry(i);
                 u64 off = composite(key_of(e.y), e.x) - lo;
                 if (off <= width) atomicAdd(&hist[(u32)(off >> s)], 1u);
             }
@@ -849,7 +893,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                     if (eck[k] - lo <= width2) gather[atomicAdd(fill, 1u)] = eck[k];
                 }
                 for (u32 i = rest; i < C; i += stride) {
-                    uint2 e = list[i];
+                    uint2 e = read_entry(i);
                     u64 ck = composite(key_of(e.y), e.x);
                     if (ck - lo <= width2) gather[atomicAdd(fill, 1u)] = ck;
                 }
@@ -975,7 +1019,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         bool pred = false;
         uint2 e = make_uint2(0, 0);
         if (i < C) {
-            e = list[i];
+            e = read_entry(i);
             pred = composite(key_of(e.y), e.x) >= T;
         }
         u32 m = __ballot_sync(0xffffffffu, pred);
