@@ -7,14 +7,16 @@
 // files it under j as it emits it (see emit_entry), in one of two ways:
 //
 //   slots   (at most kSlotWorkers workers and a slot table that fits the budget)
-//           head[j] keeps the first entry e0 to arrive: it owns the coordinate.
-//           Every later entry sets the word's top bit ("shared"), sets its worker's
-//           bit in the 128-bit mask at the start of row e0 of the table and writes
-//           its value to its worker's column of that row.  agg_reduce: an owner
-//           whose coordinate is not shared has the whole sum in its own entry; a
-//           shared one reads the mask and then the columns it names — independent
-//           loads, eight at a time — and adds them, its own value at its own
-//           worker's place, in worker order.
+//           head[j] keeps the first entry e0 to arrive: it owns the coordinate and
+//           says so in its own mark word (next[e0], one word per entry).  Every later
+//           entry marks next[e0] as shared, sets its worker's bit in the 128-bit mask
+//           at the start of row e0 of the table and writes its value to its worker's
+//           column of that row.  agg_reduce reads the marks in entry order — the
+//           coordinate words themselves, scattered over a buffer far larger than L2,
+//           are only written (back to zero).  An owner whose coordinate is not shared
+//           has the whole sum in its own entry; a shared one reads the mask and then
+//           the columns it names — independent loads, eight at a time — and adds
+//           them, its own value at its own worker's place, in worker order.
 //   chains  (otherwise)  next[e] = exchange(head[j], e+1); the entry at the head
 //           of a chain walks it — dependent loads, one per sender — and puts
 //           the terms in worker order.
@@ -49,7 +51,7 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u3
     u32 j = up[e].x;
     if (j >= d) { raise_status(ctrl, -5); next[e] = 0; return; }
     if (slots) {
-        file_in_slot(head, slots, row_words, atomicCAS(&head[j], 0u, e + 1), j, e / K_up, up[e].y);
+        file_in_slot(next, slots, row_words, atomicCAS(&head[j], 0u, e + 1), e, e / K_up, up[e].y);
     } else {
         next[e] = atomicExch(&head[j], e + 1);
     }
@@ -60,7 +62,7 @@ constexpr int kWindow = 128;  // consecutive workers whose terms one walk of a c
 // (256, 8): all 2048 threads of an SM stay resident — the kernel lives on memory parallelism
 __global__ void __launch_bounds__(256, 8)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
-                  u32* head, const u32* __restrict__ next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
+                  u32* head, u32* next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
                   int stats) {
     dependency_wait();   // the entries are filed by the kernel before
@@ -75,10 +77,16 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         own_p = p[e / K_up];  // asked for now, not after the coordinate's word has come back
         j = mine.x;
         own_bits = mine.y;
-        u32 h = j < d ? __ldcg(&head[j]) : 0u;
-        // with chains the word is a plain entry number (N*K_up < 2^31), so the mask changes nothing
-        owner = (h & 0x7fffffffu) == e + 1;
-        shared = (h >> 31) != 0;
+        if (slots) {
+            // this entry's mark says whether it owns its coordinate and whether others sent it too: no
+            // look at the coordinate's own word, which sits in a buffer far larger than L2
+            const u32 m = __ldcg(&next[e]);
+            if (m) next[e] = 0;
+            owner = (m & kMarkOwner) != 0 && j < d;
+            shared = (m & kMarkShared) != 0;
+        } else {
+            owner = j < d && __ldcg(&head[j]) == e + 1;
+        }
     }
     if (owner && slots) {
         const u32 own_q = e / K_up;

@@ -233,7 +233,7 @@ struct tk_ctx {
     SelectBufs up;             // uplink selection; up.out = the N uplink messages
     RowState* uni = nullptr;   // state of the union list / downlink selection
     u32* head = nullptr;       // [d] dense server buffer, zero at rest
-    u32* next = nullptr;       // [N*K_up]
+    u32* next = nullptr;       // [N*K_up] chain links, or (slot scheme) one mark word per entry, zero at rest
     u32* slots = nullptr;      // [N*K_up][slot_row_words] slot table, zero at rest; NULL when the server step uses chains
     u32 slot_row_words = 0;
     uint2* U = nullptr;        // [ucap] aggregate over the union
@@ -702,6 +702,7 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
               cudaMemsetAsync(c->ghist, 0, (size_t)kGridScratchWords * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemsetAsync(c->head, 0, (size_t)d * sizeof(u32), c->stream) == cudaSuccess &&
               (!c->slots || cudaMemsetAsync(c->slots, 0, L.slot_words * sizeof(u32), c->stream) == cudaSuccess) &&
+              cudaMemsetAsync(c->next, 0, (size_t)(N * K_up) * sizeof(u32), c->stream) == cudaSuccess &&
               cudaMemcpyAsync(c->p, p_host, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream) ==
                   cudaSuccess &&
               cudaStreamSynchronize(c->stream) == cudaSuccess;
@@ -726,7 +727,7 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     u32 total = (u32)(c->N * c->K_up);
     u32 blocks = (total + 255) / 256;
     int rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(256), 0, s, 0, (const uint2*)c->up.out, total,
-                              (u32)c->K_up, (const float*)c->p, c->head, (const u32*)c->next, c->slots, c->slot_row_words, c->uni, c->U,
+                              (u32)c->K_up, (const float*)c->p, c->head, c->next, c->slots, c->slot_row_words, c->uni, c->U,
                               c->ucap, w_dev,
                               scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : (float*)nullptr, c->ctrl, (u32)c->d,
                               diag ? 1 : 0);

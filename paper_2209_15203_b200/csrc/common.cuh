@@ -158,19 +158,24 @@ __device__ __forceinline__ float sq4(uint4 v, float acc) {
     return fmaf(a, a, fmaf(b, b, fmaf(c, c, fmaf(e, e, acc))));
 }
 
-// Slot filing of the server step (few workers), given what the compare-and-swap on head[idx] returned: 0 means this entry was the
-// first at the coordinate and owns it (its value stays where it is, in the message); otherwise the
-// word holds the owner's entry number + 1, and this entry marks the coordinate as shared (top bit),
-// sets its worker's bit in the 128-bit mask that opens the owner's row of the slot table and leaves
-// its value in its worker's column of that row.  Nothing here waits for a result.
-constexpr u32 kSharedBit = 0x80000000u;
+// Slot filing of the server step (few workers), given what the compare-and-swap on head[idx]
+// returned.  0: this entry e was the first at the coordinate and owns it (its value stays where it
+// is, in the message); it says so in its own word of `mark` (bit 0).  Otherwise the word holds the
+// owner's entry number + 1, and this entry marks the owner's word (bit 1: "shared"), sets its
+// worker's bit in the 128-bit mask that opens the owner's row of the slot table and leaves its
+// value in its worker's column of that row.  The marks are one word per entry (read back in entry
+// order, unlike the coordinate words, which are scattered over a buffer far larger than L2); all
+// of them are zero at rest.  Nothing here waits for a result.
+constexpr u32 kMarkOwner = 1u, kMarkShared = 2u;
 constexpr u32 kSlotMaskWords = 4;
 
-__device__ __forceinline__ void file_in_slot(u32* head, u32* slots, u32 row_words, u32 seen, u32 idx, u32 worker,
-                                             u32 bits) {
-    if (seen == 0) return;
-    if (!(seen & kSharedBit)) atomicOr(&head[idx], kSharedBit);
-    u32* row = slots + (size_t)((seen & ~kSharedBit) - 1) * row_words;
+__device__ __forceinline__ void file_in_slot(u32* mark, u32* slots, u32 row_words, u32 seen, u32 e, u32 worker, u32 bits) {
+    if (seen == 0) {
+        atomicOr(&mark[e], kMarkOwner);
+        return;
+    }
+    atomicOr(&mark[seen - 1], kMarkShared);
+    u32* row = slots + (size_t)(seen - 1) * row_words;
     atomicOr(row + (worker >> 5), 1u << (worker & 31u));
     row[kSlotMaskWords + worker] = bits;
 }

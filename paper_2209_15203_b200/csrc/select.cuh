@@ -679,9 +679,9 @@ struct LinkArgs {
     float* zero_src;
     size_t zero_stride;
     int stats;  // diagnostics: add the squares of the emitted values to RowState.sel_sq
-    // Few workers: instead of chains, head[idx] keeps the first entry e0 to arrive at the coordinate;
-    // every later entry sets the word's top bit and files its value in row e0 of the slot table
-    // (row_words words per row, all zero at rest); see aggregate.cuh.
+    // Few workers: instead of chains, head[idx] keeps the first entry e0 to arrive at the coordinate and
+    // next[] holds one mark word per entry (owner / shared); every later entry files its value in row e0
+    // of the slot table (row_words words per row, all zero at rest); see aggregate.cuh.
     u32* slots;
     u32 row_words;
 };
@@ -712,7 +712,7 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
             link.next[e] = 0;
             raise_status(ctrl, -5);
         } else if (link.slots) {
-            file_in_slot(link.head, link.slots, link.row_words, atomicCAS(&link.head[idx], 0u, e + 1), idx, link.row_base + row, bits);
+            file_in_slot(link.next, link.slots, link.row_words, atomicCAS(&link.head[idx], 0u, e + 1), e, link.row_base + row, bits);
         } else {
             link.next[e] = atomicExch(&link.head[idx], e + 1);
         }
@@ -1005,7 +1005,7 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
                     if (link.head) {
                         u32 e = (link.row_base + row) * (u32)out_stride + slot;
                         if (idx >= link.d) { link.next[e] = 0; raise_status(ctrl, -5); }
-                        else if (link.slots) file_in_slot(link.head, link.slots, link.row_words, fetched[k], idx, link.row_base + row, bits);
+                        else if (link.slots) file_in_slot(link.next, link.slots, link.row_words, fetched[k], e, link.row_base + row, bits);
                         else link.next[e] = fetched[k];
                     }
                     if (link.stats) sel_sq += (double)__uint_as_float(bits) * (double)__uint_as_float(bits);
