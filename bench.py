@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch, from the ncu capture
 # summarised under profiles/ (filter kernel, 2 of the 8 workers): (992.13 + 3.32) MB,
 # scaled by the rows of the launch (None for any other workload, or once the kernel has changed)
-FILTER_TRAFFIC_PER_ROW_CONFIG5 = (992.08e6 + 3.62e6) / 2
+FILTER_TRAFFIC_PER_ROW_CONFIG5 = (992.13e6 + 3.33e6) / 2
 
 
 def measured_hbm_gbs():
