@@ -157,3 +157,65 @@ def test_toy_example_of_the_paper():
     assert abs(norm_both - g["norm_both"][0]) < 0.03 * g["norm_both"][0]
     # both variants hover at a distance from F*, as the paper describes, far below the start
     assert F_star < F(w) < F_star + 0.2 * (F(w0) - F_star)
+
+
+def test_gap_constants_from_nonzero_memories_hand_worked():
+    # one iteration that STARTS from non-zero eps and delta (Section 3's two gap assumptions with
+    # a^q = eps^q + alpha g^q); all values by hand in the golden file
+    g = _read("gap_constants_with_memories.txt")
+    p = np.array(g["p"], np.float32)
+    K_up, K_down, alpha = int(g["K_up"][0]), int(g["K_down"][0]), g["alpha"][0]
+    G = np.array([g["g1"], g["g2"]], np.float32)
+    eps = np.array([g["eps1"], g["eps2"]], np.float32)
+    delta = np.array(g["delta"], np.float32)
+    den = g["rho_sq_den"][0]
+    uni = oracle.ref_rho(G, eps, None, K_up, K_down, p, alpha, 0)
+    bi = oracle.ref_rho(G, eps, delta, K_up, K_down, p, alpha, 1)
+    assert abs(uni - (g["rho_hat_sq_num"][0] / den) ** 0.5) < 1e-12
+    assert abs(bi - (g["rho_sq_num"][0] / den) ** 0.5) < 1e-12
+    # the unidirectional iteration has no server memory: passing one changes nothing
+    assert oracle.ref_rho(G, eps, delta, K_up, K_down, p, alpha, 0) == uni
+    # the step size sits inside a^q and in the denominator: halving it and doubling the gradients
+    # leaves every a^q, hence both ratios, unchanged
+    assert oracle.ref_rho(2 * G, eps, None, K_up, K_down, p, alpha / 2, 0) == uni
+    assert oracle.ref_rho(2 * G, eps, delta, K_up, K_down, p, alpha / 2, 1) == bi
+    # ... and the memories matter: without them the values are different ones
+    assert abs(oracle.ref_rho(G, np.zeros_like(eps), np.zeros_like(delta), K_up, K_down, p, alpha, 1) - bi) > 0.1
+
+    # second iteration of the two-iteration example (memories eps_1, delta_1 of its first iteration)
+    h = _read("alg12_two_iterations_with_memories.txt")
+    p2 = np.array(h["p"], np.float32)
+    G2 = np.array([h["g1_t2"], h["g2_t2"]], np.float32)
+    eps1 = np.array([h["eps1_t1"], h["eps2_t1"]], np.float32)
+    delta1 = np.array(h["bi_delta_t1"], np.float32)
+    K = int(h["K"][0])
+    den2 = h["rho_sq_den_t2"][0]
+    assert abs(oracle.ref_rho(G2, eps1, None, K, K, p2, h["alpha"][0], 0) - (h["rho_hat_sq_num_t2"][0] / den2) ** 0.5) < 1e-12
+    assert abs(oracle.ref_rho(G2, eps1, delta1, K, K, p2, h["alpha"][0], 1) - (h["rho_sq_num_t2"][0] / den2) ** 0.5) < 1e-12
+
+
+def test_compensated_value_takes_two_roundings():
+    # a = fl(eps + fl(alpha * g)) (first worker line of Algorithm 1/2), not a fused multiply-add.
+    # alpha = g = 1 + 2^-12: alpha*g = 1 + 2^-11 + 2^-24, which rounds (tie to even) to 1 + 2^-11;
+    # with eps = -(1 + 2^-11) the two-roundings value is exactly 0, the fused one 2^-24.
+    one_p = np.float32(1.0 + 2.0 ** -12)
+    tiny = np.float32(2.0 ** -30)
+    G = np.array([[one_p, tiny, 0.0]], np.float32)
+    eps = np.array([[-(1.0 + 2.0 ** -11), 0.0, 0.0]], np.float32)
+    p = np.ones(1, np.float32)
+    # exact products, as a check of the construction itself (float64 holds them exactly)
+    assert float(one_p) * float(one_p) == 1.0 + 2.0 ** -11 + 2.0 ** -24
+    assert np.float32(float(one_p) * float(one_p)) == np.float32(1.0 + 2.0 ** -11)
+    a1 = np.float32(float(one_p) * float(tiny))              # alpha * 2^-30, far below 2^-24
+    assert 0 < a1 < 2.0 ** -24
+    for mode in (0, 1):
+        r = oracle.ref_step_ef(np.zeros(3, np.float32), eps, np.zeros(3, np.float32), G, 1, 1, p, float(one_p), mode)
+        # coordinate 0 compensates to exactly 0, so the tiny coordinate 1 is the one sent ...
+        assert r.up_idx.tolist() == [[1]] and r.up_val[0, 0] == a1
+        # ... and what stays in the memory at coordinate 0 is exactly zero (fused: 2^-24 would be sent)
+        assert r.eps.tolist() == [[0.0, 0.0, 0.0]]
+        assert r.w.tolist() == [0.0, -float(a1), 0.0]
+    # the gap constants use the same a: Top_1(a) = {1}, Top_2(D_a) = {1, 0 (a zero)} -> difference 0;
+    # a fused a_0 = 2^-24 would be sent instead of coordinate 1 and leave a non-zero difference
+    assert oracle.ref_rho(G, eps, None, 1, 2, p, float(one_p), 0) == 0.0
+    assert oracle.ref_rho(G, eps, np.zeros(3, np.float32), 1, 2, p, float(one_p), 1) == 0.0
