@@ -52,7 +52,8 @@ enum {
     TK_ERR_INVALID = -1,  /* bad argument (range, NULL, alignment, size) */
     TK_ERR_ALLOC = -2,    /* workspace too small / allocation failed */
     TK_ERR_CUDA = -3,     /* a CUDA runtime call failed */
-    TK_ERR_TIMEOUT = -4,  /* a bounded device-side wait expired */
+    /* -4 is not used: no kernel of the library waits on a flag (all device-side waiting is a
+       cooperative-groups grid or cluster barrier), so there is no wait that could expire */
     TK_ERR_INTERNAL = -5, /* a device-side consistency check failed */
     TK_ERR_TOO_LARGE = -6 /* the problem does not fit the built-in scratch of tk_topk_noalloc */
 };
@@ -146,8 +147,14 @@ int tk_step_host(tk_ctx* ctx, float* w_host, const float* grads_host, float alph
  *   x_dev      [rows][d]
  *   idx_out_dev, val_out_dev   [rows][K], ascending index per row
  * rows, d, K need not match the context.  Scratch memory is taken from a
- * per-process pool that grows with cudaMalloc when a larger problem arrives
+ * per-device pool that grows with cudaMalloc when a larger problem arrives
  * (tk_release_scratch frees it).  Asynchronous unless the pool has to grow.
+ * The pool is one region shared by every tk_topk and tk_last_* call on the device, whatever
+ * the context: the library orders its users itself (each call makes its stream wait for the
+ * previous user's last kernel, through an event), so calls on different streams or contexts
+ * may be issued back to back from one host thread.  Two host threads must not call into the
+ * pool at the same time, and a call issued while its stream is being captured into a CUDA
+ * graph is not ordered against other users (serialise those yourself).
  */
 int tk_topk(tk_ctx* ctx, const float* x_dev, int32_t rows, int64_t d, int64_t K,
             int32_t* idx_out_dev, float* val_out_dev);
@@ -184,11 +191,17 @@ int tk_topk(tk_ctx* ctx, const float* x_dev, int32_t rows, int64_t d, int64_t K,
  *     left in it; the function clears the parts that must start at zero.  Two
  *     calls whose GPU work overlaps (different streams, different host
  *     threads) race on it: serialise them.
+ *   - The kernels' consistency checks (an entry outside its list, an empty bucket)
+ *     report into a status word in the last 256 bytes of the array.  No call clears
+ *     it, so it stays set until tk_topk_noalloc_status() reads it: that function
+ *     waits for the device (cudaDeviceSynchronize), returns the word (TK_OK or a
+ *     negative TK_ERR_* code) and puts it back to zero.  It allocates nothing either.
  * Asynchronous; results are identical to tk_topk's.
  */
 #define TK_NOALLOC_SCRATCH_BYTES (4u << 20)
 int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
                     float* val_out_dev, void* cuda_stream);
+int tk_topk_noalloc_status(void);
 
 /*
  * Error memories: the iteration exactly as Algorithm 1 / Algorithm 2 print it.
@@ -222,8 +235,12 @@ int tk_ef_state(tk_ctx* ctx, float** eps_dev, float** delta_dev);
 int tk_set_kdown(tk_ctx* ctx, int64_t K_down);
 
 /*
- * Messages of the last tk_step, for inspection.  Each call synchronises, sorts a
- * copy by index and writes it to caller-provided device buffers.
+ * Messages of the last tk_step, for inspection.  Each call synchronises, sorts the
+ * message by index and writes it to caller-provided device buffers.  The step leaves its
+ * messages in arbitrary order in the workspace and the sort permutes them there, in place
+ * (the sets do not change and nothing reads their order afterwards; the next step overwrites
+ * them).  Unlike a zero-copy accessor these calls hand out no pointer into the workspace:
+ * the caller provides the buffers and receives the entry count.
  *   tk_last_uplink     the N uplink messages, [N][K_up]
  *   tk_last_aggregate  the aggregate g as (index, value) over the union U of the
  *                      uplink index sets (g is zero elsewhere); buffers of
@@ -271,6 +288,33 @@ typedef struct tk_diag {
 int tk_set_diagnostics(tk_ctx* ctx, int level);
 int tk_diagnostics(tk_ctx* ctx, tk_diag* out, double* one_minus_gamma_up_host);
 
+/*
+ * Section 4.2's communication model of one iteration.  A sparse message costs two 32-bit words
+ * per entry (index and value).  With alpha1 / alpha2 the uplink / downlink latency and beta1 /
+ * beta2 the uplink / downlink transfer time of one 32-bit word (caller-supplied, any consistent
+ * unit of time), the paper's two formulas are
+ *     unidirectional   alpha1 + 2 K_up beta1 + alpha2 + 2 N K_up beta2
+ *     bidirectional    alpha1 + 2 K_up beta1 + alpha2 + 2 K_down beta2
+ * (the first takes the aggregate at its bound of N K_up non-zeros).
+ *   N, K_up, K_down   as for tk_init (1 <= N, 1 <= K_up, 1 <= K_down)
+ *   union_size        |U| of a step as tk_status reports it (tk_stats.union_size), 0 <= |U| <= N K_up,
+ *                     or -1 when none is known
+ * Pure host arithmetic: no context, no device.  Returns TK_ERR_INVALID for sizes out of range,
+ * negative or non-finite latencies / word times, or a NULL out.
+ */
+typedef struct tk_comm {
+    int64_t uplink_words;           /* 2 K_up: what one worker sends */
+    int64_t downlink_words_uni_max; /* 2 N K_up: the unidirectional downlink at its bound */
+    int64_t downlink_words_uni;     /* 2 |U|: what it actually carries (-1 if union_size was -1) */
+    int64_t downlink_words_bi;      /* 2 K_down */
+    double time_uni;                /* first formula */
+    double time_uni_union;          /* first formula with 2 |U| in place of 2 N K_up (-1 if union_size was -1) */
+    double time_bi;                 /* second formula */
+    double compression_factor;      /* K_down / (K_up N): downlink size after compression relative to the bound */
+} tk_comm;
+int tk_comm_model(int32_t N, int64_t K_up, int64_t K_down, int64_t union_size, double alpha1, double beta1,
+                  double alpha2, double beta2, tk_comm* out);
+
 /* Record device timestamps around the streaming selection pass of every `every`-th tk_step
  * (0 = off, 1 = every step); tk_status reports their sum.  A timestamped step is always issued
  * as plain launches, also when tk_set_graph is on. */
@@ -293,6 +337,16 @@ int tk_set_graph(tk_ctx* ctx, int on);
  * Both give identical results.
  */
 int tk_set_force_general(tk_ctx* ctx, int on);
+
+/*
+ * Testing aid (host-side fault injection): cap the candidate list every row of this context's
+ * uplink selections (tk_step, tk_step_uplink, tk_topk with this context) may use at `cap`
+ * entries (values below K are raised to K; 0 restores the capacity the workspace was laid out
+ * for).  With a cap near K every row overflows its list after the single streaming pass, fails
+ * verification and is redone by the exact multi-pass path: the results are identical, only
+ * slower.  Returns TK_ERR_INVALID for a negative cap.
+ */
+int tk_set_cand_cap(tk_ctx* ctx, int64_t cap);
 
 /* Kernels launched on the context's stream since tk_init. */
 int64_t tk_launch_count(tk_ctx* ctx);

@@ -20,10 +20,10 @@ TK_MODE_UNI = 0
 TK_MODE_BIDIR = 1
 TK_MODE_EF = 2
 
-EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_ef_bytes",
+EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_topk_noalloc_status", "tk_ef_bytes",
            "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
-           "tk_set_force_general", "tk_set_graph", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
+           "tk_set_force_general", "tk_set_cand_cap", "tk_comm_model", "tk_set_graph", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
 
 class TkError(RuntimeError):
@@ -43,6 +43,13 @@ class tk_diag(ctypes.Structure):
     _fields_ = [("nonzero_fraction", ctypes.c_double), ("union_fraction", ctypes.c_double),
                 ("compression_factor", ctypes.c_double), ("one_minus_gamma_up_max", ctypes.c_double),
                 ("one_minus_gamma_down", ctypes.c_double), ("rho", ctypes.c_double)]
+
+
+class tk_comm(ctypes.Structure):
+    _fields_ = [("uplink_words", ctypes.c_int64), ("downlink_words_uni_max", ctypes.c_int64),
+                ("downlink_words_uni", ctypes.c_int64), ("downlink_words_bi", ctypes.c_int64),
+                ("time_uni", ctypes.c_double), ("time_uni_union", ctypes.c_double), ("time_bi", ctypes.c_double),
+                ("compression_factor", ctypes.c_double)]
 
 
 _lib = None
@@ -81,6 +88,13 @@ def load(build_if_missing: bool = True):
     lib.tk_topk.argtypes = [vp, vp, i32, i64, i64, vp, vp]
     lib.tk_topk_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, vp]
     lib.tk_topk_noalloc.restype = ctypes.c_int
+    lib.tk_topk_noalloc_status.argtypes = []
+    lib.tk_topk_noalloc_status.restype = ctypes.c_int
+    lib.tk_set_cand_cap.argtypes = [vp, i64]
+    lib.tk_set_cand_cap.restype = ctypes.c_int
+    lib.tk_comm_model.argtypes = [i32, i64, i64, i64, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                  ctypes.c_double, ctypes.POINTER(tk_comm)]
+    lib.tk_comm_model.restype = ctypes.c_int
     lib.tk_ef_bytes.argtypes = [i64, i32, i64]
     lib.tk_ef_bytes.restype = ctypes.c_size_t
     lib.tk_ef_attach.argtypes = [vp, vp, ctypes.c_size_t]
@@ -276,6 +290,10 @@ class Context:
     def tk_set_force_general(self, on: bool) -> None:
         _check(load().tk_set_force_general(self._h, 1 if on else 0), "tk_set_force_general")
 
+    def tk_set_cand_cap(self, cap: int) -> None:
+        """Testing aid: cap every row's candidate list (0 restores the laid-out capacity)."""
+        _check(load().tk_set_cand_cap(self._h, int(cap)), "tk_set_cand_cap")
+
     def tk_launch_count(self) -> int:
         return int(load().tk_launch_count(self._h))
 
@@ -287,8 +305,16 @@ def tk_topk(x: torch.Tensor, K: int, ctx: Optional[Context] = None) -> Tuple[tor
     idx = torch.empty((rows, K), dtype=torch.int32, device=x.device)
     val = torch.empty((rows, K), dtype=torch.float32, device=x.device)
     with torch.cuda.device(x.device):
+        # The library runs on the context's stream, or on the legacy default stream without a
+        # context; x and the fresh outputs belong to torch's current stream.  Order the two.
+        cur = torch.cuda.current_stream(x.device)
+        run = ctx.stream if ctx is not None else torch.cuda.default_stream(x.device)
+        if run != cur:
+            run.wait_stream(cur)
         _check(load().tk_topk(ctx._h if ctx is not None else None, _dev(x2, torch.float32), rows, d, K,
                               idx.data_ptr(), val.data_ptr()), "tk_topk")
+        if run != cur:
+            cur.wait_stream(run)
     if x.dim() == 1:
         return idx[0], val[0]
     return idx, val
@@ -307,6 +333,21 @@ def tk_topk_noalloc(x: torch.Tensor, K: int, idx: torch.Tensor, val: torch.Tenso
         s = stream if stream is not None else torch.cuda.current_stream(x.device)
         _check(load().tk_topk_noalloc(_dev(x2, torch.float32), rows, d, K, _dev(idx, torch.int32),
                                       _dev(val, torch.float32), s.cuda_stream), "tk_topk_noalloc")
+
+
+def tk_comm_model(N: int, K_up: int, K_down: int, union_size: int, alpha1: float, beta1: float,
+                  alpha2: float, beta2: float) -> tk_comm:
+    """Section 4.2's words per step and transfer times (host arithmetic only; needs no GPU)."""
+    out = tk_comm()
+    _check(load().tk_comm_model(N, K_up, K_down, union_size, alpha1, beta1, alpha2, beta2, ctypes.byref(out)),
+           "tk_comm_model")
+    return out
+
+
+def tk_topk_noalloc_status() -> int:
+    """Waits for the device, then returns and clears the sticky status word of tk_topk_noalloc
+    (0, or the negative TK_ERR_* code a kernel's consistency check raised)."""
+    return int(load().tk_topk_noalloc_status())
 
 
 def tk_release_scratch() -> None:

@@ -10,7 +10,7 @@ CSRC = os.path.join(_HERE, "csrc")
 # TOPK_LIBRARY selects another build of the library (for example one compiled with different tuning macros)
 LIB = os.environ.get("TOPK_LIBRARY") or os.path.join(_HERE, "libtopk.so")
 SOURCES = ["api.cu"]
-HEADERS = ["common.cuh", "select.cuh", "sort.cuh", "aggregate.cuh"]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh"))   # every header api.cu may include
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -181,16 +181,30 @@ SortLayout sort_layout(int64_t rows, int64_t n) {
 }
 
 // ---- per-device scratch pool (tk_topk and the inspection calls) ------------------------------
+// One region per device, shared by every user whatever its stream: a user makes its stream wait
+// for the previous user's last kernel before it touches the region (pool_get) and leaves an event
+// behind its own last kernel (pool_done).
 struct Pool {
     char* base = nullptr;
     size_t bytes = 0;
+    cudaEvent_t last = nullptr;  // recorded behind the last kernel of the most recent user
+    bool pending = false;
 };
 Pool g_pool[64];
 
-int pool_get(size_t bytes, char** out) {
+bool stream_is_capturing(cudaStream_t s) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &st) != cudaSuccess) { cudaGetLastError(); return false; }
+    return st != cudaStreamCaptureStatusNone;
+}
+
+int pool_get(size_t bytes, char** out, cudaStream_t stream) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
     Pool& p = g_pool[dev];
+    if (p.pending && !stream_is_capturing(stream)) {
+        if (cudaStreamWaitEvent(stream, p.last, 0) != cudaSuccess) { cudaGetLastError(); return TK_ERR_CUDA; }
+    }
     if (p.bytes < bytes) {
         if (p.base) {
             if (cudaDeviceSynchronize() != cudaSuccess) return TK_ERR_CUDA;
@@ -210,12 +224,33 @@ int pool_get(size_t bytes, char** out) {
     return TK_OK;
 }
 
+// Call after the last kernel that uses the region has been enqueued on `stream`.
+void pool_done(cudaStream_t stream) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+    Pool& p = g_pool[dev];
+    if (stream_is_capturing(stream)) return;
+    if (!p.last && cudaEventCreateWithFlags(&p.last, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        p.last = nullptr;
+        return;
+    }
+    if (cudaEventRecord(p.last, stream) == cudaSuccess) p.pending = true;
+    else cudaGetLastError();
+}
+
 bool aligned4(const void* p) { return p != nullptr && ((uintptr_t)p & 3u) == 0; }
 
 int bits_of(int64_t v) {  // number of significant bits of v >= 0
     int b = 0;
     while (v > 0) { ++b; v >>= 1; }
     return b;
+}
+
+// Candidate capacity under tk_set_cand_cap: never above what the buffers hold, never below K.
+u32 capped(u32 laid_out, int64_t limit, int64_t K) {
+    int64_t c = limit < K ? K : limit;
+    return c < (int64_t)laid_out ? (u32)c : laid_out;
 }
 
 }  // namespace
@@ -242,6 +277,7 @@ struct tk_ctx {
     u32 ucap = 0;
     // host state
     int force_general = 0;
+    int64_t cand_cap = 0;      // tk_set_cand_cap: 0 = the capacity the workspace was laid out for
     int diagnostics = 0;
     int profile = 0;           // 0 = off, n = timestamp the streaming pass of every n-th step
     int64_t steps_seen = 0;
@@ -869,7 +905,9 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
     }
     LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0, c->slots, c->slot_row_words};
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
-    rc = run_select(s, grads_dev, c->N, c->d, c->K_up, c->up, c->ctrl, c->force_general != 0, e0, e1,
+    SelectBufs up = c->up;
+    if (c->cand_cap > 0) up.cap = capped(up.cap, c->cand_cap, c->K_up);  // shorter lists, packed closer in the same buffer
+    rc = run_select(s, grads_dev, c->N, c->d, c->K_up, up, c->ctrl, c->force_general != 0, e0, e1,
                     &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
     if (rc != TK_OK) return rc;
     rc = run_server(c, w_dev, alpha, mode);
@@ -897,6 +935,7 @@ int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_
     const bool with_ef = (mode & TK_MODE_EF) != 0;
     // this rank's slice of every per-row buffer
     SelectBufs b = c->up;
+    if (c->cand_cap > 0) b.cap = capped(b.cap, c->cand_cap, c->K_up);
     b.rs += row0;
     b.hist += (size_t)row0 * kHistBins;
     b.smax += (size_t)row0 * kSampleSlots;
@@ -959,7 +998,7 @@ int tk_topk(tk_ctx* c, const float* x_dev, int32_t rows, int64_t d, int64_t K, i
     SortLayout QL = sort_layout(rows, K);
     size_t off_ctrl = SL.bytes + QL.bytes;
     char* base = nullptr;
-    int rc = pool_get(off_ctrl + align_up(sizeof(Ctrl)), &base);
+    int rc = pool_get(off_ctrl + align_up(sizeof(Ctrl)), &base, s);
     if (rc != TK_OK) return rc;
     SelectBufs b = bind(SL, base);
     Ctrl* ctrl = c ? c->ctrl : (Ctrl*)(base + off_ctrl);
@@ -969,10 +1008,13 @@ int tk_topk(tk_ctx* c, const float* x_dev, int32_t rows, int64_t d, int64_t K, i
         return TK_ERR_CUDA;
     int64_t local = 0;
     int64_t* launches = c ? &c->launches : &local;
+    if (c && c->cand_cap > 0) b.cap = capped(b.cap, c->cand_cap, K);
     rc = run_select(s, x_dev, rows, d, K, b, ctrl, c ? c->force_general != 0 : false, nullptr, nullptr, launches);
-    if (rc != TK_OK) return rc;
-    return run_sort(s, b.out, (size_t)K, nullptr, 0, (u32)K, rows, d, (uint2*)(base + SL.bytes + QL.off_tmp),
-                    (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, launches);
+    if (rc == TK_OK)
+        rc = run_sort(s, b.out, (size_t)K, nullptr, 0, (u32)K, rows, d, (uint2*)(base + SL.bytes + QL.off_tmp),
+                      (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, launches);
+    pool_done(s);  // the next user of the pool, on whatever stream, waits for these kernels
+    return rc;
 }
 
 size_t tk_ef_bytes(int64_t d, int32_t N, int64_t K_down) {
@@ -1024,7 +1066,7 @@ int tk_last_uplink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev) {
     if (!c || !aligned4(idx_out_dev) || !aligned4(val_out_dev) || c->last_mode < 0) return TK_ERR_INVALID;
     SortLayout QL = sort_layout(c->N, c->K_up);
     char* base = nullptr;
-    int rc = pool_get(QL.bytes, &base);
+    int rc = pool_get(QL.bytes, &base, c->stream);
     if (rc != TK_OK) return rc;
     rc = run_sort(c->stream, c->up.out, (size_t)c->K_up, nullptr, 0, (u32)c->K_up, c->N, c->d,
                   (uint2*)(base + QL.off_tmp), (u32*)(base + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev,
@@ -1045,7 +1087,7 @@ int tk_last_aggregate(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64
     if (n == 0) return TK_OK;
     SortLayout QL = sort_layout(1, n);
     char* base = nullptr;
-    int rc = pool_get(QL.bytes, &base);
+    int rc = pool_get(QL.bytes, &base, c->stream);
     if (rc != TK_OK) return rc;
     rc = run_sort(c->stream, c->U, c->ucap, nullptr, 0, n, 1, c->d, (uint2*)(base + QL.off_tmp),
                   (u32*)(base + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, n, &c->launches);
@@ -1062,7 +1104,7 @@ int tk_last_downlink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64_
         u32 Kd = (u32)c->last_kdown;
         SortLayout QL = sort_layout(1, Kd);
         char* base = nullptr;
-        int rc = pool_get(QL.bytes, &base);
+        int rc = pool_get(QL.bytes, &base, c->stream);
         if (rc != TK_OK) return rc;
         *count_host = Kd;
         rc = run_sort(c->stream, c->down.out, Kd, nullptr, 0, Kd, 1, c->d, (uint2*)(base + QL.off_tmp),
@@ -1084,7 +1126,7 @@ int tk_last_downlink(tk_ctx* c, int32_t* idx_out_dev, float* val_out_dev, int64_
     size_t off_flags = off_msg + align_up((size_t)Kd * sizeof(uint2));
     size_t off_cnt = off_flags + align_up((size_t)Kd);
     char* base = nullptr;
-    int rc = pool_get(off_cnt + kAlign, &base);
+    int rc = pool_get(off_cnt + kAlign, &base, c->stream);
     if (rc != TK_OK) return rc;
     uint2* msg = (uint2*)(base + off_msg);
     unsigned char* flags = (unsigned char*)(base + off_flags);
@@ -1245,6 +1287,33 @@ int tk_set_force_general(tk_ctx* c, int on) {
     return TK_OK;
 }
 
+int tk_set_cand_cap(tk_ctx* c, int64_t cap) {
+    if (!c || cap < 0) return TK_ERR_INVALID;
+    if (cap != c->cand_cap) drop_graphs(c);  // captured steps carry the old capacity
+    c->cand_cap = cap;
+    return TK_OK;
+}
+
+int tk_comm_model(int32_t N, int64_t K_up, int64_t K_down, int64_t union_size, double alpha1, double beta1,
+                  double alpha2, double beta2, tk_comm* out) {
+    if (!out || N < 1 || K_up < 1 || K_down < 1 || (int64_t)N * K_up >= ((int64_t)1 << 31)) return TK_ERR_INVALID;
+    if (union_size < -1 || union_size > (int64_t)N * K_up) return TK_ERR_INVALID;
+    if (!isfinite(alpha1) || !isfinite(beta1) || !isfinite(alpha2) || !isfinite(beta2) || alpha1 < 0 || beta1 < 0 ||
+        alpha2 < 0 || beta2 < 0)
+        return TK_ERR_INVALID;
+    memset(out, 0, sizeof *out);
+    out->uplink_words = 2 * K_up;
+    out->downlink_words_uni_max = 2 * (int64_t)N * K_up;
+    out->downlink_words_uni = union_size < 0 ? -1 : 2 * union_size;
+    out->downlink_words_bi = 2 * K_down;
+    const double up = alpha1 + (double)out->uplink_words * beta1;
+    out->time_uni = up + alpha2 + (double)out->downlink_words_uni_max * beta2;
+    out->time_uni_union = union_size < 0 ? -1.0 : up + alpha2 + (double)out->downlink_words_uni * beta2;
+    out->time_bi = up + alpha2 + (double)out->downlink_words_bi * beta2;
+    out->compression_factor = (double)K_down / ((double)K_up * (double)N);
+    return TK_OK;
+}
+
 int64_t tk_launch_count(tk_ctx* c) { return c ? c->launches : 0; }
 
 void tk_destroy(tk_ctx* c) {
@@ -1274,18 +1343,12 @@ void tk_release_scratch(void) {
 // cudaGetSymbolAddress: the kernels get the device address looked up below.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[TK_NOALLOC_SCRATCH_BYTES];
 static char* g_noalloc_addr[64];  // device address of the array, per device; NULL until looked up
+// The last 256 bytes hold the control block with the sticky status word: zero when the library is
+// loaded (static storage), written by the kernels' consistency checks, cleared only by
+// tk_topk_noalloc_status.  Everything below it is per-call scratch.
+constexpr size_t kNoallocCtrlOff = (size_t)TK_NOALLOC_SCRATCH_BYTES - 256;
 
-int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
-                    float* val_out_dev, void* cuda_stream) {
-    if (!aligned4(x_dev) || !aligned4(idx_out_dev) || !aligned4(val_out_dev)) return TK_ERR_INVALID;
-    if (rows < 1 || d < 1 || d >= ((int64_t)1 << 31) || K < 1 || K > d) return TK_ERR_INVALID;
-    // size check first, in 64-bit arithmetic that cannot wrap for any accepted rows/d/K
-    if ((double)rows * ((double)candidate_capacity(d, K) + 2.0 * (double)K) * 8.0 > (double)TK_NOALLOC_SCRATCH_BYTES)
-        return TK_ERR_TOO_LARGE;
-    SelectLayout SL = select_layout(rows, d, K, false);
-    SortLayout QL = sort_layout(rows, K);
-    size_t off_ctrl = SL.bytes + QL.bytes;
-    if (off_ctrl + align_up(sizeof(Ctrl)) > (size_t)TK_NOALLOC_SCRATCH_BYTES) return TK_ERR_TOO_LARGE;
+static int noalloc_base(char** out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
     if (!g_noalloc_addr[dev]) {  // set-up, once per device, with that device current
@@ -1296,20 +1359,53 @@ int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int3
         }
         g_noalloc_addr[dev] = (char*)ptr;
     }
-    char* base = g_noalloc_addr[dev];
+    *out = g_noalloc_addr[dev];
+    return TK_OK;
+}
+
+int tk_topk_noalloc(const float* x_dev, int32_t rows, int64_t d, int64_t K, int32_t* idx_out_dev,
+                    float* val_out_dev, void* cuda_stream) {
+    if (!aligned4(x_dev) || !aligned4(idx_out_dev) || !aligned4(val_out_dev)) return TK_ERR_INVALID;
+    if (rows < 1 || d < 1 || d >= ((int64_t)1 << 31) || K < 1 || K > d) return TK_ERR_INVALID;
+    // size check first, in 64-bit arithmetic that cannot wrap for any accepted rows/d/K
+    if ((double)rows * ((double)candidate_capacity(d, K) + 2.0 * (double)K) * 8.0 > (double)kNoallocCtrlOff)
+        return TK_ERR_TOO_LARGE;
+    SelectLayout SL = select_layout(rows, d, K, false);
+    SortLayout QL = sort_layout(rows, K);
+    if (SL.bytes + QL.bytes > kNoallocCtrlOff) return TK_ERR_TOO_LARGE;
+    char* base = nullptr;
+    int rc = noalloc_base(&base);
+    if (rc != TK_OK) return rc;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     SelectBufs b = bind(SL, base);
-    Ctrl* ctrl = (Ctrl*)(base + off_ctrl);
+    Ctrl* ctrl = (Ctrl*)(base + kNoallocCtrlOff);
     // the array still holds the previous call's data: clear what the kernels expect to be zero
+    // (not the control block: its status word is sticky)
     if (cudaMemsetAsync(b.rs, 0, (size_t)rows * sizeof(RowState), s) != cudaSuccess ||
-        cudaMemsetAsync(b.hist, 0, (size_t)rows * kHistBins * sizeof(u32), s) != cudaSuccess ||
-        cudaMemsetAsync(ctrl, 0, sizeof(Ctrl), s) != cudaSuccess)
+        cudaMemsetAsync(b.hist, 0, (size_t)rows * kHistBins * sizeof(u32), s) != cudaSuccess)
         return TK_ERR_CUDA;
     int64_t launches = 0;
-    int rc = run_select(s, x_dev, rows, d, K, b, ctrl, false, nullptr, nullptr, &launches);
+    rc = run_select(s, x_dev, rows, d, K, b, ctrl, false, nullptr, nullptr, &launches);
     if (rc != TK_OK) return rc;
     return run_sort(s, b.out, (size_t)K, nullptr, 0, (u32)K, rows, d, (uint2*)(base + SL.bytes + QL.off_tmp),
                     (u32*)(base + SL.bytes + QL.off_cnt), QL.tiles, idx_out_dev, val_out_dev, (size_t)K, &launches);
+}
+
+int tk_topk_noalloc_status(void) {
+    char* base = nullptr;
+    int rc = noalloc_base(&base);
+    if (rc != TK_OK) return rc;
+    Ctrl ctrl;  // on the stack: nothing is allocated here either
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(&ctrl, base + kNoallocCtrlOff, sizeof ctrl, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    if (ctrl.status != 0 && cudaMemset(base + kNoallocCtrlOff, 0, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return ctrl.status;
 }
 
 const char* tk_strerror(int code) {
@@ -1318,7 +1414,6 @@ const char* tk_strerror(int code) {
         case TK_ERR_INVALID: return "invalid argument";
         case TK_ERR_ALLOC: return "workspace too small or allocation failed";
         case TK_ERR_CUDA: return "CUDA runtime error";
-        case TK_ERR_TIMEOUT: return "bounded device-side wait expired";
         case TK_ERR_INTERNAL: return "device-side consistency check failed";
         case TK_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of tk_topk_noalloc";
         default: return "unknown error";

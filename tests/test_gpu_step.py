@@ -108,6 +108,30 @@ def test_scaled_configs_forced_general_path():
     run_workload(W.workload(4, d=500_000, N=6), 2, force_general=True)
 
 
+def test_forced_list_overflow_redoes_every_row_exactly():
+    # host-side fault injection: with the candidate lists capped just above K every row of an ordinary
+    # input overflows its list in the streaming pass, fails verification and is redone by the exact
+    # multi-pass path; the results are the oracle's all the same
+    for wl in (W.workload(2, d=600_001, N=4), W.workload(3, d=700_002, N=5)):
+        ctx = make_ctx(wl, wl.K_down[0])
+        w_dev = W.make_w(wl, DEV)
+        w_ref = w_dev.cpu().numpy()
+        for s, cap in enumerate((wl.K_up + 5, 1, 0, wl.K_up)):     # 1 is raised to K; 0 restores the full lists
+            ctx.tk_set_cand_cap(cap)
+            G = W.make_grads(wl, s, DEV)
+            w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, 1, wl.K_down[0], "capped lists cap=%d" % cap)
+            st = ctx.tk_status()
+            assert st.rows_general == (0 if cap == 0 else wl.N), (cap, st.rows_general)
+        # the standalone selection with the same context obeys the cap too
+        ctx.tk_set_cand_cap(wl.K_up + 1)
+        G = W.make_grads(wl, 9, DEV)
+        idx, val = ctx.tk_topk(G, wl.K_up)
+        ref_idx, ref_val = oracle.ref_topk_rows(G.cpu().numpy(), wl.K_up)
+        assert_message_equal(idx, val, ref_idx, ref_val, "tk_topk with capped lists")
+        assert ctx.tk_status().rows_general == wl.N
+        ctx.close()
+
+
 def test_kdown_larger_than_union_pads_with_zero_entries():
     wl = W.workload(4, d=400_000, N=4)          # K_up = 40, union <= 160; K_down = 4000 > |U|
     assert wl.K_down[-1] > wl.N * wl.K_up
@@ -389,11 +413,14 @@ def _host_can_hold(wl):
     return psutil.virtual_memory().available > need * 1.2
 
 
-@pytest.mark.parametrize("cid,steps", [(2, 2), (3, 1), (4, 1), (5, 1)])
-def test_full_size_configs(cid, steps):
+@pytest.mark.parametrize("cid,steps,mode,kdowns", [(2, 2, 1, None), (3, 1, 1, None), (3, 1, 0, None), (4, 1, 1, (0, 2)),
+                                                   (4, 1, 1, (1,)), (5, 1, 1, None)])
+def test_full_size_configs(cid, steps, mode, kdowns):
+    # every leg the five configurations name, a slice of its steps each (the opt-in acceptance run
+    # of test_gpu_acceptance.py does all steps): config 3 in both modes, config 4 at its three K_down
     wl = W.workload(cid)
     if not _host_can_hold(wl):
         pytest.skip("not enough host memory for the oracle at this size")
-    if cid == 4:
-        wl = wl.__class__(**{**wl.__dict__, "K_down": (wl.K_down[0], wl.K_down[2])})
-    run_workload(wl, steps, modes=(1,))
+    if kdowns is not None:
+        wl = wl.__class__(**{**wl.__dict__, "K_down": tuple(wl.K_down[i] for i in kdowns)})
+    run_workload(wl, steps, modes=(mode,))
