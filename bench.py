@@ -32,10 +32,50 @@ METRIC = "gradient elements/sec per bidirectional top_K step"
 UNIT = "elements/s"
 NOMINAL_HBM_BPS = 8e12
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one filter_kernel launch, from the ncu capture
-# summarised under profiles/ (filter kernel, 2 of the 8 workers): (992.13 + 3.32) MB,
-# scaled by the rows of the launch (None for any other workload, or once the kernel has changed)
-FILTER_TRAFFIC_PER_ROW_CONFIG5 = (992.13e6 + 3.33e6) / 2
+PROFILE_SUMMARY = os.path.join(ROOT, "profiles", "filter_kernel_config5_rows2.md")
+KERNEL_SOURCES = ["paper_2209_15203_b200/csrc/common.cuh", "paper_2209_15203_b200/csrc/select.cuh"]
+
+
+def kernel_source_digest():
+    """sha256 over the sources of the streaming kernel (what decides whether captured counters still apply)."""
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def captured_traffic(path=PROFILE_SUMMARY):
+    """The `key: value` lines of the ncu summary of the streaming kernel: DRAM bytes read + written per
+    launch, the rows that launch covered and the digest of the kernel sources it was taken on."""
+    import re
+    out = {}
+    try:
+        with open(path) as f:
+            for line in f:
+                m = re.match(r"^\s*(dram_bytes_read_per_launch|dram_bytes_write_per_launch|rows_per_launch|"
+                             r"kernel_source_sha256)\s*:\s*(\S+)\s*$", line)
+                if m:
+                    out[m.group(1)] = m.group(2)
+    except OSError:
+        return None
+    if len(out) != 4:
+        return None
+    return {"read": float(out["dram_bytes_read_per_launch"]), "write": float(out["dram_bytes_write_per_launch"]),
+            "rows": int(out["rows_per_launch"]), "sha256": out["kernel_source_sha256"]}
+
+
+def traffic_for(wl, overridden_d, ef):
+    """DRAM traffic of one launch of the streaming kernel on the benchmark workload, scaled by rows from
+    the captured case (traffic is proportional to the rows); None for any other workload, and None once
+    the kernel sources differ from the ones the counters were taken on."""
+    if wl.cid != 5 or overridden_d or ef:
+        return None
+    cap = captured_traffic()
+    if cap is None or cap["sha256"] != kernel_source_digest():
+        return None
+    return (cap["read"] + cap["write"]) / cap["rows"] * wl.N
 
 
 def measured_hbm_gbs():
@@ -104,49 +144,63 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+def sum_checksum(t):
+    """workloads.checksum row by row (bounded temporary memory), wrapped to 64 bits."""
+    total = 0
+    for q in range(t.shape[0]):
+        total = (total + W.checksum(t[q])) & 0xFFFFFFFFFFFFFFFF
+    return total
+
+
 def b_min_bytes(wl, k_apply):
     return 4 * wl.N * wl.d + 24 * wl.N * wl.K_up + 16 * k_apply
 
 
+REFERENCE_BUDGET_S = 300.0   # wall-clock the reference arm may spend inside the oracle
+
+
 def run_reference(args, rank, world):
-    """The CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    """The CPU oracle, as it stands, on the host cores (rank 0 only): full steps of the stated
+    configuration (same N, d, K as the GPU arm).  A full step of the largest workload costs the oracle
+    about 20 s, so what is bounded is the NUMBER of steps run and timed, never the problem: one warm-up
+    step, then as many of the requested steps as fit REFERENCE_BUDGET_S (at least one)."""
     if rank != 0:
         return
     import oracle
-    wl_full = W.workload(args.config)
-    threads = min(wl_full.N, oracle.ref.default_threads())
-    total_steps = args.steps + args.warmup
-    # a full step of the largest workload costs the oracle roughly 2e-8 s per element on 8 cores;
-    # shrink d so that the whole run stays within a few minutes
-    budget = 150.0 / max(1, total_steps)
-    d = wl_full.d
-    est = 2.0e-8 * wl_full.N * d
-    if est > budget:
-        d = max(200_000, int(d * budget / est) // 1000 * 1000)
-    wl = W.workload(args.config, d=d)
+    wl = W.workload(args.config)
+    threads = min(wl.N, oracle.ref.default_threads())
     p = W.make_p(wl).numpy()
-    scale = W.scale_vector(wl, "cpu")
     w = W.make_w(wl, "cpu").numpy()
     K_down = wl.K_down[0]
+    # one gradient tensor for all steps (generating 4 GB on the host costs as much as a step; the
+    # oracle's time does not depend on the values, and w still changes from step to step)
+    G = W.make_grads(wl, 0, "cpu", agree=args.agree).numpy()
     times = []
-    for s in range(total_steps):
-        G = W.make_grads(wl, s, "cpu", scale=scale, agree=args.agree).numpy()
+    spent = 0.0
+    n_warm = 1 if args.warmup > 0 else 0
+    s = 0
+    while True:
         t0 = time.perf_counter()
         res = oracle.ref_step(w, G, wl.K_up, K_down, p, wl.alpha, 1, nthreads=threads, want_dense=False)
-        t1 = time.perf_counter()
+        dt = time.perf_counter() - t0
         w = res.w
-        if s >= args.warmup:
-            times.append(t1 - t0)
+        spent += dt
+        if s >= n_warm:
+            times.append(dt)
+        s += 1
+        if len(times) >= args.steps or (times and spent + dt > REFERENCE_BUDGET_S):
+            break
     t = sum(times)
     value = wl.N * wl.d * len(times) / t
-    sample = "config %d recipe at d=%d of %d (N=%d, K=%d), full steps" % (wl.cid, wl.d, wl_full.d, wl.N, wl.K_up)
-    cfg = W.describe(wl_full)
-    cfg["sampled_d"] = wl.d
+    ts = sorted(times)
+    sample = ("%d full steps of config %d timed (of %d asked; N=%d rows of d=%d, K=%d) after %d warm-up, "
+              "%.0f s in the oracle" % (len(times), wl.cid, args.steps, wl.N, wl.d, wl.K_up, n_warm, spent))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / len(times),
+        "steps": args.steps, "warmup": args.warmup, "steps_timed": len(times), "warmup_run": n_warm,
+        "ms_per_step": 1e3 * t / len(times), "ms_per_step_median": 1e3 * ts[len(ts) // 2], "ms_per_step_min": 1e3 * ts[0],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": cfg,
+        "config": W.describe(wl),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -251,14 +305,17 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = ctx.tk_launch_count()
     barrier()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]   # one behind every step
     sampler.start()
     ev0.record()
     for s in range(args.steps):
         step(bufs[s % nbuf])
+        marks[s].record()
     ev1.record()
     barrier()
     sampler.stop_flag = True
     ms = ev0.elapsed_time(ev1)
+    per_step = sorted(a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks))
     launches = ctx.tk_launch_count() - launches0
     st = ctx.tk_status()
     sampler.join(timeout=2.0)
@@ -278,10 +335,16 @@ def main():
         bytes_per_elem = 12.0 if args.ef else 4.0   # with memories: read g, read and write epsilon
         elems_rank = (elems // world) if args.sharded else elems     # what one launch on this rank reads
         achieved = bytes_per_elem * elems_rank / (k_ms * 1e-3) / 1e9
+        step_bytes = b_min_bytes(wl, K_down) + (8 * elems + 4 * wl.d if args.ef else 0)
+        step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
         roof = {"bound": "hbm", "kernel": "filter_kernel" if st.rows_general == 0 else "general_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": FILTER_TRAFFIC_PER_ROW_CONFIG5 * wl.N if (wl.cid == 5 and not args.d and not args.ef) else None,
-                "algorithmic_bytes": int(bytes_per_elem) * elems_rank, "kernel_ms": k_ms, "launches_timed": st.select_samples}
+                "peak_note": "a read+write copy; a read-only stream can exceed it slightly",
+                "traffic": traffic_for(wl, args.d, args.ef),
+                "algorithmic_bytes": int(bytes_per_elem) * elems_rank, "kernel_ms": k_ms, "launches_timed": st.select_samples,
+                # the whole step (all kernels, minimum bytes of the method) against the same peak and the nominal one
+                "whole_step": {"algorithmic_bytes": step_bytes, "achieved": step_gbs, "frac": step_gbs / peak,
+                               "frac_of_nominal_8TBps": step_gbs * 1e9 / NOMINAL_HBM_BPS}}
 
     # end to end through tk_step_host: pinned host buffers, copies inside the timed region
     e2e = None
@@ -319,8 +382,13 @@ def main():
         else:
             oracle.ref_step(w_cpu, G, wl.K_up, K_down, p.numpy(), wl.alpha, 1, nthreads=threads, want_dense=False)
         dt = time.perf_counter() - t0
+        # ... and Top_K of one row on one thread (the unit of work the rows are spread over)
+        t0 = time.perf_counter()
+        oracle.ref_topk(G[0], wl.K_up)
+        dt_row = time.perf_counter() - t0
         cpu = {"value": elems / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": "1 full step of config %d (N=%d rows of d=%d), %.1f s" % (wl.cid, wl.N, wl.d, dt)}
+               "sample": "1 full step of config %d (N=%d rows of d=%d), %.1f s" % (wl.cid, wl.N, wl.d, dt),
+               "one_row_topk_single_thread_s": dt_row, "one_row_topk_single_thread_elements_per_s": wl.d / dt_row}
 
     if rank == 0:
         cfg = W.describe(wl)
@@ -332,15 +400,28 @@ def main():
                                     else "replicas x%d") % world})
         if args.agree is not None:
             cfg["rows"] = "shared vector x (1 + %g z_q)" % args.agree
+        cfg["input_checksum_step0"] = "%016x" % sum_checksum(bufs[0])
+        # Section 4.2's transfer model for this workload.  beta = one 32-bit word at the 770 GB/s a peer copy
+        # reaches on this pool's NVLink (from the pool's measurements, not this run); latencies are not
+        # measurable on one GPU and are left at 0, so the times are the bandwidth terms alone.
+        beta = 4.0 / 770e9
+        cm = binding.tk_comm_model(wl.N, wl.K_up, K_down, int(st.union_size), 0.0, beta, 0.0, beta)
+        comm = {"uplink_words_per_worker": cm.uplink_words, "downlink_words_uni_bound": cm.downlink_words_uni_max,
+                "downlink_words_uni_last_step": cm.downlink_words_uni, "downlink_words_bi": cm.downlink_words_bi,
+                "compression_factor": cm.compression_factor,
+                "alpha_s": 0.0, "beta_s_per_word": beta, "time_uni_s": cm.time_uni, "time_uni_union_s": cm.time_uni_union,
+                "time_bi_s": cm.time_bi, "note": "beta assumed from the pool's peer-copy rate, latencies not measured"}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "warmup": warmup, "ms_per_step": ms_per_step,
+            "ms_per_step_median": per_step[len(per_step) // 2], "ms_per_step_min": per_step[0],
+            "higher_is_better": True,
             "scaling": "strong" if args.sharded else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
             "hbm_frac_of_8TBps": (b_min_bytes(wl, K_down) + (8 * elems + 4 * wl.d if args.ef else 0))
             / (ms_per_step * 1e-3) / NOMINAL_HBM_BPS,
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": sampler.summary(),
+            "clocks": sampler.summary(), "comm_model": comm,
             "stats": {"rows_general": st.rows_general, "union_size": st.union_size,
                       "cand_min": st.cand_min, "cand_max": st.cand_max, "device_status": st.device_status},
         }
