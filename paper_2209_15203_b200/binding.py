@@ -23,7 +23,7 @@ TK_MODE_EF = 2
 EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_topk_noalloc_status", "tk_ef_bytes",
            "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
-           "tk_set_force_general", "tk_set_cand_cap", "tk_comm_model", "tk_set_graph", "tk_launch_count", "tk_destroy", "tk_release_scratch", "tk_strerror"]
+           "tk_set_force_general", "tk_set_cand_cap", "tk_comm_model", "tk_set_graph", "tk_launch_count", "tk_debug_phase_clock", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
 
 class TkError(RuntimeError):
@@ -116,6 +116,8 @@ def load(build_if_missing: bool = True):
     lib.tk_set_graph.restype = ctypes.c_int
     lib.tk_launch_count.argtypes = [vp]
     lib.tk_launch_count.restype = i64
+    lib.tk_debug_phase_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), ctypes.c_int32]
+    lib.tk_debug_phase_clock.restype = ctypes.c_int
     lib.tk_destroy.argtypes = [vp]
     lib.tk_destroy.restype = None
     lib.tk_release_scratch.argtypes = []
@@ -296,6 +298,21 @@ class Context:
 
     def tk_launch_count(self) -> int:
         return int(load().tk_launch_count(self._h))
+
+    PHASE_STAMPS = ("sampling starts", "sampling ends", "streaming pass starts", "streaming pass ends",
+                    "fused kernel starts", "rows verified", "uplink selected", "barrier passed", "aggregated",
+                    "barrier passed", "done", "uplink: candidates loaded", "uplink: first level done",
+                    "uplink: threshold known", "downlink: entries loaded", "downlink: first level done",
+                    "downlink: threshold known", "uplink: output slots known", "uplink: coordinate words answered")
+
+    def tk_debug_phase_clock(self):
+        """(first_us, last_us) per stamp of PHASE_STAMPS for the last step, and re-arms the stamps.
+        Needs a library built with -DTK_PHASE_CLOCK=1 (raises otherwise)."""
+        n = len(self.PHASE_STAMPS)
+        first = (ctypes.c_double * n)()
+        last = (ctypes.c_double * n)()
+        _check(load().tk_debug_phase_clock(self._h, first, last, n), "tk_debug_phase_clock")
+        return list(first), list(last)
 
 
 def tk_topk(x: torch.Tensor, K: int, ctx: Optional[Context] = None) -> Tuple[torch.Tensor, torch.Tensor]:

@@ -42,7 +42,7 @@ constexpr int kPredictLightTurns = 2;  // ... in the variant for many rows
 #endif
 constexpr int kFilterThreads = TK_FILTER_THREADS;  // filter kernel: threads per CTA
 constexpr int kFilterCtasPerSm = TK_FILTER_CTAS;   // filter kernel: resident CTAs per SM (grid = that x SMs)
-constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads per CTA
+constexpr int kGeneralThreads = 1024;              // multi-pass phase: threads per CTA (the block shape of the fused kernel)
 constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
 constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
@@ -86,7 +86,23 @@ struct RowState {
     double sum_sq;   // sum of squares of the whole vector
     double sel_sq;   // sum of squares of the emitted entries
     u32 nnz;         // union list: entries whose value is not zero
-    u32 min_key;     // union list: smallest key among its entries (lower end of the downlink selection's first range)
+    u32 pad_;
+};
+
+// Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the
+// nanosecond global timer) at their phase boundaries; tk_debug_phase_clock reads them.  Off in
+// the ordinary build: the stamps cost an atomic per CTA and phase.
+#ifndef TK_PHASE_CLOCK
+#define TK_PHASE_CLOCK 0
+#endif
+enum : int {
+    kStampPredictStart = 0, kStampPredictEnd, kStampFilterStart, kStampFilterEnd, kStampTailStart, kStampVerified,
+    kStampSelected, kStampSelectedAll, kStampAggregated, kStampAggregatedAll, kStampDone,
+    // inside the uplink (per row) and the downlink selection: candidates in registers, first
+    // level's bucket found, threshold known
+    kStampUpLoaded, kStampUpLevel, kStampUpThreshold, kStampDownLoaded, kStampDownLevel, kStampDownThreshold,
+    kStampUpSlots, kStampUpFetched,  // uplink emission: output slots known, coordinate words answered
+    kStampCount
 };
 
 // Step-wide control block.
@@ -94,7 +110,21 @@ struct Ctrl {
     int status;        // sticky TK_ERR_* raised on the device
     u32 rows_general;  // rows the multi-pass path handled in the last selection
     u32 pad[6];
+#if TK_PHASE_CLOCK
+    u64 t_first[kStampCount];  // earliest / latest time any CTA passed each stamp
+    u64 t_last[kStampCount];
+#endif
 };
+
+// One thread per CTA calls.
+__device__ __forceinline__ void phase_stamp(Ctrl* ctrl, int which) {
+#if TK_PHASE_CLOCK
+    u64 t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(&ctrl->t_first[which], t);
+    atomicMax(&ctrl->t_last[which], t);
+#endif
+}
 
 __device__ __forceinline__ u32 key_of(u32 bits) { return bits & 0x7fffffffu; }
 
