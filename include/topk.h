@@ -352,16 +352,15 @@ int tk_set_cand_cap(tk_ctx* ctx, int64_t cap);
 int64_t tk_launch_count(tk_ctx* ctx);
 
 /*
- * Developer aid, no counterpart in the paper: device timestamps at the phase boundaries of the
- * last step.  Only a library compiled with -DTK_PHASE_CLOCK=1 records them (every CTA then does
- * two atomics per phase); the ordinary build returns TK_ERR_INVALID.  Synchronises.  For each
- * of the first n stamps (sampling start / end, streaming pass start / end, start of the fused
- * kernel after it, rows verified, uplink selected, barrier passed, aggregated, barrier passed,
- * done; then, inside the uplink and the downlink selection: entries loaded, first level done,
- * threshold known; uplink emission: output slots known, coordinate words answered:
- * 19 in all) first_us / last_us [n] (host) receive the earliest and the latest time any
- * CTA passed it, in microseconds since the earliest stamp, -1 where no CTA passed.  The call
- * then re-arms the stamps, so call it once before the step to be measured.
+ * Developer aid, no counterpart in the paper: device timestamps of the last step's kernels.
+ * Only a library compiled with -DTK_PHASE_CLOCK=1 records them (every CTA then does two atomics
+ * per stamp); the ordinary build returns TK_ERR_INVALID.  Synchronises.  For each of the first n
+ * stamps first_us / last_us [n] (host) receive the earliest and the latest time any CTA passed
+ * it, in microseconds since the earliest stamp, -1 where no CTA passed.  The 18 stamps, in order:
+ * sampling starts / ends; streaming pass starts / ends; verification starts / ends; uplink
+ * selection: starts (its predecessors have ended), candidates loaded, first level done,
+ * threshold known, ends; server sum starts / ends; downlink selection: the same five.
+ * The call then re-arms the stamps, so call it once before the step to be measured.
  */
 int tk_debug_phase_clock(tk_ctx* ctx, double* first_us, double* last_us, int32_t n);
 

@@ -300,10 +300,12 @@ class Context:
         return int(load().tk_launch_count(self._h))
 
     PHASE_STAMPS = ("sampling starts", "sampling ends", "streaming pass starts", "streaming pass ends",
-                    "fused kernel starts", "rows verified", "uplink selected", "barrier passed", "aggregated",
-                    "barrier passed", "done", "uplink: candidates loaded", "uplink: first level done",
-                    "uplink: threshold known", "downlink: entries loaded", "downlink: first level done",
-                    "downlink: threshold known", "uplink: output slots known", "uplink: coordinate words answered")
+                    "verification starts", "verification ends",
+                    "uplink select starts", "uplink: candidates loaded", "uplink: first level done",
+                    "uplink: threshold known", "uplink select ends",
+                    "server sum starts", "server sum ends",
+                    "downlink select starts", "downlink: entries loaded", "downlink: first level done",
+                    "downlink: threshold known", "downlink select ends")
 
     def tk_debug_phase_clock(self):
         """(first_us, last_us) per stamp of PHASE_STAMPS for the last step, and re-arms the stamps.

@@ -59,233 +59,164 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u3
 
 constexpr int kWindow = 128;  // consecutive workers whose terms one walk of a chain gathers (two 64-bit masks)
 
-constexpr int kAggPerThread = 4;  // entries a thread of the server phase handles per round (their loads overlap)
-
-// Shared memory of agg_phase (for CTAs of up to 1024 threads).
-struct AggShared {
-    u32 scratch[33];
-    u32 base;
-    u32 queue_n;
-    u32 hist[kHistBins];                 // keys of this CTA's sums by their leading 11 bits (first level of the downlink selection)
-    u32 queue[1024 * kAggPerThread];     // this round's owners of shared coordinates (position within the round)
-    float sum[1024 * kAggPerThread];     // ... and their sums, by the same position
-};
-
-// g_j = sum over the senders of coordinate j of fl(p_q * v_q), in worker order, for the entry e that
-// owns the coordinate (worker own_q, value own_bits); puts the words it used back to zero.
-__device__ __forceinline__ float agg_owner_sum(u32 e, u32 own_q, u32 own_bits, bool shared, const uint2* up, u32 total,
-                                               u32 K_up, const float* __restrict__ p, u32* next, u32* slots, u32 row_words) {
-    float acc = 0.0f;
-    if (slots) {
-        if (!shared) return __fadd_rn(acc, __fmul_rn(p[own_q], __uint_as_float(own_bits)));
-        u32* row = slots + (size_t)e * row_words;
-        const uint4 m = __ldcg(reinterpret_cast<const uint4*>(row));
-        u64 m0 = (u64)m.x | ((u64)m.y << 32), m1 = (u64)m.z | ((u64)m.w << 32);
-        if (own_q < 64u) m0 |= 1ull << own_q;
-        else m1 |= 1ull << (own_q - 64u);
-        while (m0 | m1) {
-            u32 qs[8], vs[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {  // the next eight senders, their values all requested at once
-                qs[i] = 0xffffffffu;
-                if (m0) { qs[i] = (u32)__ffsll((long long)m0) - 1u; m0 &= m0 - 1; }
-                else if (m1) { qs[i] = (u32)__ffsll((long long)m1) + 63u; m1 &= m1 - 1; }
-                vs[i] = 0;
-                if (qs[i] == own_q) vs[i] = own_bits;
-                else if (qs[i] != 0xffffffffu) vs[i] = __ldcg(row + kSlotMaskWords + qs[i]);
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (qs[i] == 0xffffffffu) continue;
-                acc = __fadd_rn(acc, __fmul_rn(p[qs[i]], __uint_as_float(vs[i])));
-                if (qs[i] != own_q) row[kSlotMaskWords + qs[i]] = 0;
-            }
-        }
-        *reinterpret_cast<uint4*>(row) = make_uint4(0, 0, 0, 0);
-        return acc;
-    }
-    // chains
-    // Entry ids grow with the worker (e = q*K_up + slot) and a worker sends a coordinate at most
-    // once.  A walk of the chain is a string of dependent loads, the expensive part; each hop
-    // also fetches the entry's value, so the two latencies overlap.  The values of the workers
-    // in a window of kWindow consecutive numbers go into a small table with a bit mask saying
-    // which are present; the terms are then added in ascending worker order.  With at most
-    // kWindow workers that is a single walk; with more, one walk finds the first sender and
-    // one walk per window that has senders follows.
-    u32 byv[kWindow];
-    u32 qlo = 0;  // workers below qlo are done
-    if (total > (u32)kWindow * K_up) {
-        u32 min_id = e;
-        for (u32 c = next[e], hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) min_id = min(min_id, c - 1);
-        qlo = min_id / K_up;
-    }
-    for (u32 guard = 0; guard <= total; ++guard) {
-        u64 m0 = 0, m1 = 0;
-        u32 qnext = 0xffffffffu;
-        for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; ++hops) {
-            const u32 id = c - 1;
-            const u32 nx = next[id];
-            const u32 v = __ldcg(&up[id].y);
-            const u32 q = id / K_up;
-            if (q >= qlo) {
-                const u32 o = q - qlo;
-                if (o < (u32)kWindow) {
-                    byv[o] = v;
-                    if (o < 64u) m0 |= 1ull << o;
-                    else m1 |= 1ull << (o - 64u);
-                } else {
-                    qnext = min(qnext, q);
-                }
-            }
-            c = nx;
-        }
-        while (m0) {
-            const int b = __ffsll((long long)m0) - 1;
-            m0 &= m0 - 1;
-            acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
-        }
-        while (m1) {
-            const int b = __ffsll((long long)m1) + 63;
-            m1 &= m1 - 1;
-            acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
-        }
-        if (qnext == 0xffffffffu) break;
-        qlo = qnext;
-    }
-    return acc;
-}
-
-// The server sum over all `total` entries of the message buffer, by the whole grid (every thread
-// of every CTA calls).  Per round a thread takes kAggPerThread entries, a whole grid's width
-// apart, and asks for all their words at once.  An entry that owns a coordinate nobody else sent
-// has its sum at hand (p_q * v).  The owners of shared coordinates — whose sums cost two or more
-// dependent round trips to memory — are first collected in a queue and then taken one per
-// thread, so that those round trips run side by side instead of one entry after the other.
-// The union list is appended to once per CTA and round.
-// level0, when given (kHistBins words, zero on entry): the sums' keys are also counted by their
-// leading 11 bits — the first level of the downlink selection, ready when this returns and the
-// grid has synchronised.
-template <int kThreads>
-__device__ __forceinline__ void agg_phase(AggShared& sh, const uint2* up, u32 total, u32 K_up, const float* __restrict__ p,
-                                          u32* head, u32* next, u32* slots, u32 row_words,
-                                          RowState* uni /* the union's state */, uint2* U, u32 ucap, float* w, float alpha,
-                                          int apply, float* delta, Ctrl* ctrl, u32 d, int stats, u32* level0) {
-    constexpr int R = kAggPerThread;
-    static_assert(kThreads <= 1024, "AggShared is sized for 1024 threads");
+// (256, 8): all 2048 threads of an SM stay resident — the kernel lives on memory parallelism
+__global__ void __launch_bounds__(256, 8)
+agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
+                  u32* head, u32* next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
+                  uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
+                  int stats, u32* level0) {
+    // level0, when given (kHistBins words of global memory, zero on entry): the sums' keys are also
+    // counted by their leading 11 bits — the first level of the downlink selection, complete when
+    // this grid ends
+    __shared__ u32 sh_hist[kHistBins];
     if (level0)
-        for (int b = threadIdx.x; b < kHistBins; b += kThreads) sh.hist[b] = 0;
-    const u32 width = gridDim.x * (u32)kThreads;       // entries one value of k covers
-    for (u32 round0 = 0; round0 < total; round0 += width * R) {   // u32: total < 2^31 and a round is far smaller
-        const u32 e0 = round0 + blockIdx.x * (u32)kThreads + threadIdx.x;
-        if (threadIdx.x == 0) sh.queue_n = 0;
-        __syncthreads();
-        uint2 mine[R];
-        u32 mark[R];
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            const u32 e = e0 + (u32)k * width;
-            mine[k] = make_uint2(0xffffffffu, 0u);
-            mark[k] = 0;
-            if (e < total) {
-                // written earlier in the same launch when the step is fused: L2, not the read-only path
-                mine[k] = __ldcg(&up[e]);
-                // slots: this entry's mark says whether it owns its coordinate and whether others sent it
-                // too — no look at the coordinate's own word, which sits in a buffer far larger than L2.
-                // chains: the entry's link (non-zero: others sent the coordinate before it)
-                mark[k] = __ldcg(&next[e]);
-            }
-        }
-        if (!slots) {  // chains: the owner is the entry the coordinate's word names
-#pragma unroll
-            for (int k = 0; k < R; ++k) {
-                const u32 e = e0 + (u32)k * width;
-                const bool owner = e < total && mine[k].x < d && __ldcg(&head[mine[k].x]) == e + 1;
-                mark[k] = owner ? (kMarkOwner | (mark[k] ? kMarkShared : 0u)) : 0u;
-            }
-        }
-        u32 owners_mine = 0;
-        float acc[R];
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            const u32 e = e0 + (u32)k * width;
-            acc[k] = 0.0f;
-            if (slots && mark[k]) next[e] = 0;
-            const bool owner = (mark[k] & kMarkOwner) != 0 && mine[k].x < d;
-            mark[k] = owner ? mark[k] : 0u;
-            const bool queued = owner && (mark[k] & kMarkShared) != 0;
-            if (owner) {
-                ++owners_mine;
-                if (!queued) acc[k] = __fadd_rn(0.0f, __fmul_rn(p[e / K_up], __uint_as_float(mine[k].y)));
-            }
-            // one counter update per warp
-            const u32 m = __ballot_sync(0xffffffffu, queued);
-            if (m) {
-                u32 at = 0;
-                const int leader = __ffs(m) - 1;
-                if ((int)lane_id() == leader) at = atomicAdd(&sh.queue_n, (u32)__popc(m));
-                at = __shfl_sync(0xffffffffu, at, leader);
-                if (queued) sh.queue[at + (u32)__popc(m & ((1u << lane_id()) - 1u))] = (u32)k * kThreads + threadIdx.x;
-            }
-        }
-        __syncthreads();
-        for (u32 i = threadIdx.x; i < sh.queue_n; i += kThreads) {
-            const u32 pos = sh.queue[i];
-            const u32 e = round0 + blockIdx.x * (u32)kThreads + (pos / kThreads) * width + (pos % kThreads);
-            const u32 own_bits = __ldcg(&up[e].y);
-            sh.sum[pos] = agg_owner_sum(e, e / K_up, own_bits, true, up, total, K_up, p, next, slots, row_words);
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            if (!mark[k]) continue;
-            if (mark[k] & kMarkShared) acc[k] = sh.sum[(u32)k * kThreads + threadIdx.x];
-            const u32 j = mine[k].x;
-            head[j] = 0;
-            if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc[k]));
-            // server memory (Algorithm 2): g = sum + delta, kept in the memory until the downlink
-            // selection takes its Top_K out of it
-            if (delta) delta[j] = __fadd_rn(acc[k], delta[j]);
-        }
-        if (level0) {
-#pragma unroll
-            for (int k = 0; k < R; ++k) {
-                // the sums crowd into a few bins: one shared-memory atomic per distinct bin and warp
-                const bool live = mark[k] != 0;
-                const u32 bin = key_of(__float_as_uint(acc[k])) >> 20;
-                const u32 peers = __match_any_sync(0xffffffffu, live ? bin : 0xffffffffu);
-                if (live && (int)lane_id() == __ffs(peers) - 1) atomicAdd(&sh.hist[bin], (u32)__popc(peers));
-            }
-        }
-        // append the (j, g_j) to the union list: one counter update per CTA and round
-        u32 owners;
-        u32 incl = block_inclusive_scan(owners_mine, sh.scratch, &owners);
-        if (threadIdx.x == 0 && owners) sh.base = atomicAdd(&uni->cand_count, owners);
-        __syncthreads();
-        u32 slot = sh.base + incl - owners_mine;
-        u32 nz = 0;
-        double sq = 0.0;
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            if (mark[k]) {
-                const u32 bits = __float_as_uint(acc[k]);
-                if (slot < ucap) U[slot] = make_uint2(mine[k].x, bits);
-                ++slot;
-                if (stats) {
-                    nz += key_of(bits) != 0 ? 1u : 0u;
-                    sq += (double)acc[k] * (double)acc[k];
-                }
-            }
-        }
-        if (stats) {  // diagnostics: non-zeros of the aggregate (Section 4.2) and its squared norm
-            nz = __reduce_add_sync(0xffffffffu, nz);
-            if (lane_id() == 0 && nz) atomicAdd(&uni->nnz, nz);
-            warp_add_double(&uni->sum_sq, sq);
+        for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
+    dependency_wait();   // the entries are filed by the kernel before
+    if (threadIdx.x == 0) phase_stamp(ctrl, kStampAggStart);
+    u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+    bool owner = false;
+    u32 j = 0, own_bits = 0;
+    float acc = 0.0f;
+    bool shared = false;
+    float own_p = 0.0f;
+    if (e < total) {
+        uint2 mine = up[e];
+        own_p = p[e / K_up];  // asked for now, not after the coordinate's word has come back
+        j = mine.x;
+        own_bits = mine.y;
+        if (slots) {
+            // this entry's mark says whether it owns its coordinate and whether others sent it too: no
+            // look at the coordinate's own word, which sits in a buffer far larger than L2
+            const u32 m = __ldcg(&next[e]);
+            if (m) next[e] = 0;
+            owner = (m & kMarkOwner) != 0 && j < d;
+            shared = (m & kMarkShared) != 0;
+        } else {
+            owner = j < d && __ldcg(&head[j]) == e + 1;
         }
     }
+    if (owner && slots) {
+        const u32 own_q = e / K_up;
+        if (!shared) {
+            acc = __fadd_rn(acc, __fmul_rn(own_p, __uint_as_float(own_bits)));
+        } else {
+            u32* row = slots + (size_t)e * row_words;
+            const uint4 m = __ldcg(reinterpret_cast<const uint4*>(row));
+            u64 m0 = (u64)m.x | ((u64)m.y << 32), m1 = (u64)m.z | ((u64)m.w << 32);
+            if (own_q < 64u) m0 |= 1ull << own_q;
+            else m1 |= 1ull << (own_q - 64u);
+            while (m0 | m1) {
+                u32 qs[8], vs[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {  // the next eight senders, their values all requested at once
+                    qs[i] = 0xffffffffu;
+                    if (m0) { qs[i] = (u32)__ffsll((long long)m0) - 1u; m0 &= m0 - 1; }
+                    else if (m1) { qs[i] = (u32)__ffsll((long long)m1) + 63u; m1 &= m1 - 1; }
+                    vs[i] = 0;
+                    if (qs[i] == own_q) vs[i] = own_bits;
+                    else if (qs[i] != 0xffffffffu) vs[i] = __ldcg(row + kSlotMaskWords + qs[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (qs[i] == 0xffffffffu) continue;
+                    acc = __fadd_rn(acc, __fmul_rn(p[qs[i]], __uint_as_float(vs[i])));
+                    if (qs[i] != own_q) row[kSlotMaskWords + qs[i]] = 0;
+                }
+            }
+            *reinterpret_cast<uint4*>(row) = make_uint4(0, 0, 0, 0);
+        }
+    } else if (owner) {  // chains
+        // Entry ids grow with the worker (e = q*K_up + slot) and a worker sends a coordinate at most
+        // once.  A walk of the chain is a string of dependent loads, the expensive part; each hop
+        // also fetches the entry's value, so the two latencies overlap.  The values of the workers
+        // in a window of kWindow consecutive numbers go into a small table with a bit mask saying
+        // which are present; the terms are then added in ascending worker order.  With at most
+        // kWindow workers that is a single walk; with more, one walk finds the first sender and
+        // one walk per window that has senders follows.
+        u32 byv[kWindow];
+        u32 qlo = 0;  // workers below qlo are done
+        if (total > (u32)kWindow * K_up) {
+            u32 min_id = e;
+            for (u32 c = next[e], hops = 0; c != 0 && hops <= total; c = next[c - 1], ++hops) min_id = min(min_id, c - 1);
+            qlo = min_id / K_up;
+        }
+        for (u32 guard = 0; guard <= total; ++guard) {
+            u64 m0 = 0, m1 = 0;
+            u32 qnext = 0xffffffffu;
+            for (u32 c = e + 1, hops = 0; c != 0 && hops <= total; ++hops) {
+                const u32 id = c - 1;
+                const u32 nx = next[id];
+                const u32 v = up[id].y;
+                const u32 q = id / K_up;
+                if (q >= qlo) {
+                    const u32 o = q - qlo;
+                    if (o < (u32)kWindow) {
+                        byv[o] = v;
+                        if (o < 64u) m0 |= 1ull << o;
+                        else m1 |= 1ull << (o - 64u);
+                    } else {
+                        qnext = min(qnext, q);
+                    }
+                }
+                c = nx;
+            }
+            while (m0) {
+                const int b = __ffsll((long long)m0) - 1;
+                m0 &= m0 - 1;
+                acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
+            }
+            while (m1) {
+                const int b = __ffsll((long long)m1) + 63;
+                m1 &= m1 - 1;
+                acc = __fadd_rn(acc, __fmul_rn(p[qlo + (u32)b], __uint_as_float(byv[b])));
+            }
+            if (qnext == 0xffffffffu) break;
+            qlo = qnext;
+        }
+    }
+    if (owner) {
+        head[j] = 0;
+        if (apply) w[j] = __fsub_rn(w[j], __fmul_rn(alpha, acc));
+        // server memory (Algorithm 2): g = sum + delta, kept in the memory until the downlink
+        // selection takes its Top_K out of it
+        if (delta) delta[j] = __fadd_rn(acc, delta[j]);
+    }
+    // append (j, g_j) to the union list: one counter update per CTA (every entry of every worker
+    // passes through here; per-warp atomics on the one word would serialise)
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_base;
+    u32 bits = __float_as_uint(acc);
+    u32 owners;
+    u32 incl = block_inclusive_scan(owner ? 1u : 0u, sh_scratch, &owners);
     if (level0) {
+        // the sums crowd into a few bins: one shared-memory atomic per distinct bin and warp
+        // (the scan above has passed a barrier since sh_hist was cleared)
+        const u32 bin = key_of(bits) >> 20;
+        const u32 peers = __match_any_sync(0xffffffffu, owner ? bin : 0xffffffffu);
+        if (owner && (int)lane_id() == __ffs(peers) - 1) atomicAdd(&sh_hist[bin], (u32)__popc(peers));
+    } else if (ucap <= 4096u) {
+        // a union this small is selected from by a single CTA, which wants the largest aggregated
+        // magnitude as the upper end of its first range instead of the counts
+        u32 wm = __reduce_max_sync(0xffffffffu, owner ? key_of(bits) : 0u);
+        if (lane_id() == 0 && wm) atomicMax(&uni->max_key, wm);
+    }
+    if (threadIdx.x == 0 && owners) sh_base = atomicAdd(&uni->cand_count, owners);
+    __syncthreads();
+    if (owner) {
+        u32 slot = sh_base + incl - 1;
+        if (slot < ucap) U[slot] = make_uint2(j, bits);
+    }
+    if (level0)
+        for (int b = threadIdx.x; b < kHistBins; b += blockDim.x)
+            if (sh_hist[b]) atomicAdd(&level0[b], sh_hist[b]);
+    if (stats) {  // diagnostics: non-zeros of the aggregate (Section 4.2) and its squared norm
+        u32 nz = __reduce_add_sync(0xffffffffu, (owner && key_of(bits) != 0) ? 1u : 0u);
+        if (lane_id() == 0 && nz) atomicAdd(&uni->nnz, nz);
+        warp_add_double(&uni->sum_sq, owner ? (double)acc * (double)acc : 0.0);
+    }
+    if (TK_PHASE_CLOCK) {
         __syncthreads();
-        for (int b = threadIdx.x; b < kHistBins; b += kThreads)
-            if (sh.hist[b]) atomicAdd(&level0[b], sh.hist[b]);
+        if (threadIdx.x == 0) phase_stamp(ctrl, kStampAggEnd);
     }
 }
 

@@ -13,7 +13,6 @@
 #include "diag.cuh"
 #include "select.cuh"
 #include "sort.cuh"
-#include "tail.cuh"
 
 using namespace tk;
 
@@ -27,7 +26,8 @@ size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct DeviceInfo {
     bool ready = false;
     int sms = 0;
-    int tail_grid[4] = {0, 0, 0, 0};  // co-resident CTAs of tail_kernel launched in clusters of 1, 2, 4, 8
+    int general_grid = 0;  // co-resident CTAs of general_kernel
+    int select_grid = 0;   // co-resident CTAs of the grid-wide select_kernel
 };
 DeviceInfo g_dev[64];
 
@@ -36,33 +36,17 @@ int device_info(DeviceInfo** out) {
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return TK_ERR_CUDA;
     DeviceInfo& di = g_dev[dev];
     if (!di.ready) {
-        int coop = 0;
+        int coop = 0, per_sm = 0;
         if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TK_ERR_CUDA;
         if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return TK_ERR_CUDA;
-        if (cudaFuncSetAttribute(tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TailShared)) != cudaSuccess)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, general_kernel, kGeneralThreads, 0) != cudaSuccess ||
+            per_sm < 1)
             return TK_ERR_CUDA;
-        for (int i = 0; i < 4; ++i) {
-            int cs = 1 << i, clusters = 0;
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)(di.sms / cs * cs));
-            cfg.blockDim = dim3(kTailThreads);
-            cfg.dynamicSmemBytes = sizeof(TailShared);
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = (unsigned)cs;
-            attr[0].val.clusterDim.y = 1;
-            attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            if (cudaOccupancyMaxActiveClusters(&clusters, tail_kernel, &cfg) != cudaSuccess) {
-                cudaGetLastError();
-                clusters = 0;
-            }
-            int ctas = clusters * cs;
-            if (ctas > di.sms / cs * cs) ctas = di.sms / cs * cs;  // one CTA per SM by design
-            di.tail_grid[i] = ctas;
-        }
-        if (di.tail_grid[0] < 1) return TK_ERR_CUDA;
+        di.general_grid = per_sm * di.sms;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel<true, false>, kSelectThreads, 0) != cudaSuccess ||
+            per_sm < 1)
+            return TK_ERR_CUDA;
+        di.select_grid = per_sm * di.sms;
         di.ready = true;
     }
     *out = &di;
@@ -390,20 +374,20 @@ CtxLayout ctx_layout(int64_t d, int64_t N, int64_t K_up) {
 // CTAs per row of the cluster select: the kernel issues a fixed string of instructions per
 // register-held candidate and level, so few candidates per thread (about 4) on many SMs beats
 // many per thread on few; at least 4 CTAs when there are few rows, but never so many that the
-// clusters of all rows stop being resident together (then clusters take rows in turn).
-int cluster_size_for(int64_t entries, int64_t rows, const DeviceInfo& di) {
-    int64_t per_cta = (int64_t)kSelectThreads * kSelectPerThread;
+// clusters of all rows stop fitting in one wave.
+int cluster_size_for(int64_t entries, int64_t rows, int sms) {
+    // few rows (their clusters of 8 fill at most half the SMs): half as many candidates per thread — measured
+    // on 8 rows of 25-35k candidates, clusters of 8 select 2 us faster than clusters of 4; on 16 rows 4 us slower
+    const int per_thread = rows * 16 <= sms ? (kSelectPerThread + 1) / 2 : kSelectPerThread;
+    int64_t per_cta = (int64_t)kSelectThreads * per_thread;
     int64_t need = (entries + per_cta - 1) / per_cta;
     int cs_need = 1;
     while (cs_need < 8 && cs_need < need) cs_need *= 2;
     int cs_fill = 1;
-    for (int i = 3; i > 0; --i)
-        if ((int64_t)(1 << i) * rows <= di.tail_grid[i]) { cs_fill = 1 << i; break; }
+    while (cs_fill < 8 && (int64_t)cs_fill * 2 * rows <= sms) cs_fill *= 2;
     int floor4 = cs_fill < 4 ? cs_fill : 4;
     int cs = cs_need > floor4 ? cs_need : floor4;
-    cs = cs < cs_fill ? cs : cs_fill;
-    while (cs > 1 && di.tail_grid[cs == 8 ? 3 : cs == 4 ? 2 : 1] < cs) cs /= 2;
-    return cs;
+    return cs < cs_fill ? cs : cs_fill;
 }
 
 #ifndef TK_PDL
@@ -448,39 +432,12 @@ int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
         if (cudaGetLastError() != cudaSuccess) return TK_ERR_CUDA; \
     } while (0)
 
-// The fused kernel after the streaming pass: cooperative (its phases are separated by grid-wide
-// barriers), in clusters of cs CTAs, as many CTAs as are resident together.
-int launch_tail(cudaStream_t stream, int cs, const DeviceInfo& di, const TailArgs& args) {
-    int idx = cs == 8 ? 3 : cs == 4 ? 2 : cs == 2 ? 1 : 0;
-    int grid = di.tail_grid[idx];
-    if (grid < cs) return TK_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kTailThreads);
-    cfg.dynamicSmemBytes = sizeof(TailShared);
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[3];
-    int n = 0;
-    attr[n].id = cudaLaunchAttributeCooperative;
-    attr[n].val.cooperative = 1;
-    ++n;
-    attr[n].id = cudaLaunchAttributeClusterDimension;
-    attr[n].val.clusterDim.x = (unsigned)cs;
-    attr[n].val.clusterDim.y = 1;
-    attr[n].val.clusterDim.z = 1;
-    ++n;
-    if (TK_PDL) {
-        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[n].val.programmaticStreamSerializationAllowed = 1;
-        ++n;
-    }
-    cfg.attrs = attr;
-    cfg.numAttrs = (unsigned)n;
-    if (cudaLaunchKernelEx(&cfg, tail_kernel, args) != cudaSuccess) {
-        cudaGetLastError();
-        return TK_ERR_CUDA;
-    }
-    return TK_OK;
+int launch_select(cudaStream_t stream, int rows, int cs, const uint2* lists, size_t list_stride, u32 cap,
+                  RowState* rs, u32 K, uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl) {
+    u32* no_ghist = nullptr;
+    DenseArgs no_dense = {nullptr, nullptr, 0};
+    return launch_dependent(select_kernel<false, false>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, lists,
+                            list_stride, cap, rs, K, out, out_stride, apply, link, ctrl, no_ghist, no_dense, 0);
 }
 
 // CTAs per row when the selection reads short rows directly: enough to keep (nearly) the whole row in
@@ -498,9 +455,29 @@ int dense_cluster_size(int64_t d, int64_t rows, int sms) {
 // The same selection straight from short rows (no candidate lists, no bound).
 int launch_select_dense(cudaStream_t stream, int rows, int cs, const float* x, int64_t d, RowState* rs, u32 K, uint2* out,
                         ApplyArgs apply, LinkArgs link, Ctrl* ctrl, RowState* also_reset, bool stats) {
+    u32* no_ghist = nullptr;
+    const uint2* no_lists = nullptr;
     DenseArgs dense = {x, also_reset, stats ? 1 : 0};
-    return launch_dependent(select_dense_kernel, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, (size_t)d,
-                            (u32)d, rs, K, out, apply, link, ctrl, dense);
+    return launch_dependent(select_kernel<false, true>, dim3((unsigned)(rows * cs)), dim3(kSelectThreads), 0, stream, cs, no_lists,
+                            (size_t)d, (u32)d, rs, K, out, (size_t)K, apply, link, ctrl, no_ghist, dense, 0);
+}
+
+// One long list selected by the whole grid (cooperative launch).
+int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap, RowState* rs, u32 K, uint2* out,
+                       ApplyArgs apply, Ctrl* ctrl, u32* ghist, bool stats, bool first_level_counted) {
+    size_t stride = cap;
+    LinkArgs nolink = {nullptr, nullptr, 0, 0, nullptr, 0, stats ? 1 : 0};
+    DenseArgs no_dense = {nullptr, nullptr, 0};
+    int prebuilt = first_level_counted ? 1 : 0;  // the server sum has counted the first level into ghist
+    void* args[] = {(void*)&list, (void*)&stride, (void*)&cap, (void*)&rs,  (void*)&K,    (void*)&out,
+                    (void*)&stride, (void*)&apply, (void*)&nolink, (void*)&ctrl, (void*)&ghist, (void*)&no_dense,
+                    (void*)&prebuilt};
+    if (cudaLaunchCooperativeKernel((void*)select_kernel<true, false>, dim3(ctas), dim3(kSelectThreads), args, 0, stream) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return TK_ERR_CUDA;
+    }
+    return TK_OK;
 }
 
 // Exact Top_K of every row of x into b.out ([rows][K], arbitrary order).  ev0/ev1, when
@@ -509,16 +486,10 @@ int launch_select_dense(cudaStream_t stream, int rows, int cs, const float* x, i
 // With error memories (ef.eps != NULL) the vector selected from is a = eps + alpha*x, which
 // also replaces eps; the streaming pass computes it on the fly when x and eps are equally
 // aligned, otherwise a separate pass does and the selection then reads eps alone.
-//
-// `server`, when given, holds the arguments of the phases that follow the uplink selection in a
-// step (server sum, downlink selection); they then run in the same launch as the selection's
-// last kernel and *server_fused is set.  Not possible when the rows take several launches or
-// are selected straight from short rows: the caller launches those phases itself then.
 int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
                Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches,
                RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0},
-               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}, bool stats = false,
-               const TailArgs* server = nullptr, bool* server_fused = nullptr) {
+               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}, bool stats = false) {
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
@@ -617,36 +588,33 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             TK_LAUNCH_CHECK();
             *launches += 1;
         }
-        // verification (or, without a prediction, the exact multi-pass selection) and the cluster select
-        // of every row, in one cooperative launch
-        TailArgs t = {};
-        const bool fuse = server != nullptr && rows <= kMaxRowsPerLaunch;
-        if (fuse) t = *server;
-        t.phases |= kPhaseVerify | kPhaseSelect;
-        t.ctrl = ctrl;
-        t.x = xb;
-        t.rows = nr;
-        t.d = d;
-        t.K = (u32)K;
-        t.tpr = b.tpr_general;
-        t.cap = b.cap;
-        t.rs = rs;
-        t.hist = hist;
-        t.cand = cand;
-        t.out = out;
-        t.apply_up = apply;
-        t.link = link;
-        t.link.row_base = (u32)r0;
-        t.link.stats = stats ? 1 : 0;
-        if (t.link.zero_src) t.link.zero_src += (size_t)r0 * t.link.zero_stride;
-        t.stats = stats ? 1 : 0;
+        {
+            u32 Ku = (u32)K, tpr = b.tpr_general, cap = b.cap;
+            int st = stats ? 1 : 0;
+            void* args[] = {(void*)&xb, (void*)&nr, (void*)&d, (void*)&Ku, (void*)&tpr, (void*)&cap,
+                            (void*)&rs,  (void*)&hist, (void*)&cand, (void*)&ctrl, (void*)&st};
+            // without a prediction the multi-pass kernel is the streaming pass that gets timed
+            if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
+            // no more CTAs than tiles: a grid-wide barrier costs more the more CTAs take part
+            u64 gtiles = (u64)nr * b.tpr_general;
+            unsigned ggrid = (unsigned)(gtiles < (u64)di->general_grid ? gtiles : (u64)di->general_grid);
+            if (ggrid < 1) ggrid = 1;
+            if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(ggrid), dim3(kGeneralThreads), args,
+                                            0, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return TK_ERR_CUDA;
+            }
+            if (!predict && ev1 && r0 == 0) cudaEventRecord(ev1, stream);
+            *launches += 1;
+        }
         int64_t expect = predict ? 2 * K : (int64_t)b.cap;
-        // without a prediction the multi-pass phase is the streaming pass that gets timed
-        if (!predict && ev0 && r0 == 0) cudaEventRecord(ev0, stream);
-        rc = launch_tail(stream, cluster_size_for(expect, nr, *di), *di, t);
+        LinkArgs lk = link;
+        lk.row_base = (u32)r0;
+        lk.stats = stats ? 1 : 0;
+        if (lk.zero_src) lk.zero_src += (size_t)r0 * lk.zero_stride;
+        rc = launch_select(stream, nr, cluster_size_for(expect, nr, di->sms), cand, b.cap, b.cap, rs, (u32)K, out, (size_t)K, apply,
+                           lk, ctrl);
         if (rc != TK_OK) return rc;
-        if (!predict && ev1 && r0 == 0) cudaEventRecord(ev1, stream);
-        if (fuse && server_fused) *server_fused = true;
         *launches += 1;
     }
     return TK_OK;
@@ -791,52 +759,31 @@ int tk_init(tk_ctx** out, int64_t d, int32_t N, int64_t K_up, int64_t K_down, co
 
 namespace {
 
-// Arguments of the server phases of a step (stages 2-4 on the messages in c->up.out, every entry
-// already filed under its coordinate): the ordered sum over the union and, when bidirectional
-// without memories, the downlink selection with the update.
-TailArgs server_args(tk_ctx* c, float* w_dev, float alpha, int mode) {
-    const bool bidir = (mode & TK_MODE_BIDIR) != 0, with_ef = (mode & TK_MODE_EF) != 0;
-    TailArgs t = {};
-    t.phases = kPhaseAggregate | ((bidir && !with_ef) ? kPhaseDownlink : 0);
-    t.ctrl = c->ctrl;
-    t.stats = c->diagnostics != 0 ? 1 : 0;
-    t.up = c->up.out;
-    t.total = (u32)(c->N * c->K_up);
-    t.K_up = (u32)c->K_up;
-    t.p = c->p;
-    t.head = c->head;
-    t.next = c->next;
-    t.slots = c->slots;
-    t.row_words = c->slot_row_words;
-    t.uni = c->uni;
-    t.U = c->U;
-    t.ucap = c->ucap;
-    t.w = w_dev;
-    t.alpha = with_ef ? 1.0f : alpha;  // with memories the step size is already inside the messages
-    t.apply_uni = bidir ? 0 : 1;
-    t.delta = (bidir && with_ef) ? c->delta : nullptr;
-    t.d32 = (u32)c->d;
-    t.K_down = (u32)c->K_down;
-    t.sel = c->sel;
-    t.apply_down = ApplyArgs{w_dev, alpha};
-    t.ghist = c->ghist;
-    return t;
-}
-
-// What follows the server phases.  `launched`: they already ran inside the uplink selection's launch.
-int run_server(tk_ctx* c, float* w_dev, float alpha, int mode, bool launched) {
+// Stages 2-4 on the messages in c->up.out (already threaded onto their chains).
+int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     const bool bidir = (mode & TK_MODE_BIDIR) != 0, with_ef = (mode & TK_MODE_EF) != 0;
     const bool diag = c->diagnostics != 0;
     cudaStream_t s = c->stream;
-    int rc = TK_OK;
-    if (!launched) {
-        DeviceInfo* di = nullptr;
-        rc = device_info(&di);
-        if (rc != TK_OK) return rc;
-        rc = launch_tail(s, 1, *di, server_args(c, w_dev, alpha, mode));
-        if (rc != TK_OK) return rc;
-        c->launches += 1;
-    }
+    // with memories the step size is already inside the messages
+    const float scale = with_ef ? 1.0f : alpha;
+    u32 total = (u32)(c->N * c->K_up);
+    u32 blocks = (total + 255) / 256;
+    DeviceInfo* di = nullptr;
+    int rc = device_info(&di);
+    if (rc != TK_OK) return rc;
+    // the downlink selection: the union can hold up to ucap entries, about 4096 per CTA, at most one
+    // co-resident wave.  With more than one CTA its first level is counted by the server sum already.
+    int ctas = (int)((c->ucap + 4095) / 4096);
+    if (ctas > di->select_grid) ctas = di->select_grid;
+    if (ctas < 1) ctas = 1;
+    const bool prebuilt = bidir && !with_ef && ctas > 1;
+    rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(256), 0, s, 0, (const uint2*)c->up.out, total,
+                              (u32)c->K_up, (const float*)c->p, c->head, c->next, c->slots, c->slot_row_words, c->uni, c->U,
+                              c->ucap, w_dev,
+                              scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : (float*)nullptr, c->ctrl, (u32)c->d,
+                              diag ? 1 : 0, prebuilt ? c->ghist : (u32*)nullptr);
+    if (rc != TK_OK) return rc;
+    c->launches += 1;
     if (bidir && with_ef) {
         // Algorithm 2 with the server memory: delta now holds g = sum + delta everywhere; take
         // Top_K_down out of it (delta <- g - Top_K(g)) and apply it (w <- w - Top_K(g))
@@ -845,6 +792,11 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode, bool launched) {
         rc = run_select(s, c->delta, 1, c->d, c->K_down, c->down, c->ctrl, c->force_general != 0, nullptr, nullptr,
                         &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag);
         if (rc != TK_OK) return rc;
+    } else if (bidir) {
+        ApplyArgs ap = {w_dev, alpha};
+        rc = launch_select_grid(s, ctas, c->U, c->ucap, c->uni, (u32)c->K_down, c->sel, ap, c->ctrl, c->ghist, diag, prebuilt);
+        if (rc != TK_OK) return rc;
+        c->launches += 1;
     }
     c->last_mode = mode;
     c->last_kdown = c->K_down;
@@ -963,12 +915,10 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
     SelectBufs up = c->up;
     if (c->cand_cap > 0) up.cap = capped(up.cap, c->cand_cap, c->K_up);  // shorter lists, packed closer in the same buffer
-    const TailArgs server = server_args(c, w_dev, alpha, mode);
-    bool server_fused = false;
     rc = run_select(s, grads_dev, c->N, c->d, c->K_up, up, c->ctrl, c->force_general != 0, e0, e1,
-                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag, &server, &server_fused);
+                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
     if (rc != TK_OK) return rc;
-    rc = run_server(c, w_dev, alpha, mode, server_fused);
+    rc = run_server(c, w_dev, alpha, mode);
     if (rc != TK_OK || !gap) return rc;
     // after the step: the other side of the difference is what the server actually sent
     const uint2* other = c->U;                      // unidirectional: S over the union
@@ -1020,7 +970,7 @@ int tk_step_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
                                                                  c->slot_row_words, c->uni, c->ctrl, (u32)c->d);
     TK_LAUNCH_CHECK();
     c->launches += 1;
-    return run_server(c, w_dev, alpha, mode, false);
+    return run_server(c, w_dev, alpha, mode);
 }
 
 int tk_step_host(tk_ctx* c, float* w_host, const float* grads_host, float alpha, int mode) {

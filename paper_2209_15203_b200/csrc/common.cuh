@@ -42,7 +42,7 @@ constexpr int kPredictLightTurns = 2;  // ... in the variant for many rows
 #endif
 constexpr int kFilterThreads = TK_FILTER_THREADS;  // filter kernel: threads per CTA
 constexpr int kFilterCtasPerSm = TK_FILTER_CTAS;   // filter kernel: resident CTAs per SM (grid = that x SMs)
-constexpr int kGeneralThreads = 1024;              // multi-pass phase: threads per CTA (the block shape of the fused kernel)
+constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads per CTA
 constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
 constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
@@ -57,6 +57,10 @@ constexpr int kFilterEfTileVecs = kFilterThreads * kFilterEfUnroll;
 // The filter grid splits the tile space into ranges shared by at least this many CTAs each
 // (8 ranges on 296 CTAs; 37 ranges of 8 CTAs measured 3 % slower on the 32-row workload).
 constexpr int kFilterMinCpp = TK_FILTER_MIN_CPP;
+#ifndef TK_FILTER_DYN_TILES
+#define TK_FILTER_DYN_TILES 16
+#endif
+constexpr int kFilterDynTiles = TK_FILTER_DYN_TILES;  // tiles per CTA (on average) left to be claimed at the end of a tile range; 0: none
 constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 #ifndef TK_SELECT_PER_THREAD
 #define TK_SELECT_PER_THREAD 8
@@ -86,22 +90,22 @@ struct RowState {
     double sum_sq;   // sum of squares of the whole vector
     double sel_sq;   // sum of squares of the emitted entries
     u32 nnz;         // union list: entries whose value is not zero
-    u32 pad_;
+    u32 tile_ticket; // streaming pass: tiles handed out so far from the claimed end of tile range number <this row's index>
 };
 
 // Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the
-// nanosecond global timer) at their phase boundaries; tk_debug_phase_clock reads them.  Off in
-// the ordinary build: the stamps cost an atomic per CTA and phase.
+// nanosecond global timer) where they start and end and at the milestones of the selections;
+// tk_debug_phase_clock reads them.  Off in the ordinary build: a stamp costs two atomics per CTA.
 #ifndef TK_PHASE_CLOCK
 #define TK_PHASE_CLOCK 0
 #endif
 enum : int {
-    kStampPredictStart = 0, kStampPredictEnd, kStampFilterStart, kStampFilterEnd, kStampTailStart, kStampVerified,
-    kStampSelected, kStampSelectedAll, kStampAggregated, kStampAggregatedAll, kStampDone,
-    // inside the uplink (per row) and the downlink selection: candidates in registers, first
-    // level's bucket found, threshold known
-    kStampUpLoaded, kStampUpLevel, kStampUpThreshold, kStampDownLoaded, kStampDownLevel, kStampDownThreshold,
-    kStampUpSlots, kStampUpFetched,  // uplink emission: output slots known, coordinate words answered
+    kStampPredictStart = 0, kStampPredictEnd, kStampFilterStart, kStampFilterEnd, kStampVerifyStart, kStampVerifyEnd,
+    // a selection: its predecessors have ended, candidates in registers, first level's bucket found,
+    // threshold known, everything emitted
+    kStampUpStart, kStampUpLoaded, kStampUpLevel, kStampUpThreshold, kStampUpEnd,
+    kStampAggStart, kStampAggEnd,
+    kStampDownStart, kStampDownLoaded, kStampDownLevel, kStampDownThreshold, kStampDownEnd,
     kStampCount
 };
 

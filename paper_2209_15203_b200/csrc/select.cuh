@@ -47,6 +47,7 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->out_count = 0;
     r->flags = flags;
     r->ticket = 0;
+    r->tile_ticket = 0;
     r->g_active = 0;
     r->sum_sq = 0.0;
     r->sel_sq = 0.0;
@@ -206,9 +207,6 @@ __device__ __forceinline__ RowGeom row_geom(const float* x, int row, int64_t d) 
 #ifndef TK_STAGE_SLOTS
 #define TK_STAGE_SLOTS 128
 #endif
-#ifndef TK_FILTER_TRIGGER
-#define TK_FILTER_TRIGGER 1
-#endif
 constexpr int kStageSlots = TK_STAGE_SLOTS;  // per warp; at least 32 (128 measured 0.3-0.7 % faster per step than 64)
 
 struct WarpStage {
@@ -310,12 +308,12 @@ __device__ __forceinline__ bool may_hit(uint4 v, float thr) {
 // zeroed there by the selection's emission: eps <- a - Top_K(a)).
 // With kStats the squares of all values of the tile are added to `sq` (per thread, fp32).
 template <int THREADS, int UNROLL, bool kEF, bool kStats>
-__device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u32 tid, u64 lo, const WarpStage& st,
+__device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u64 lo, const WarpStage& st,
                                             RowState* rs, uint2* cand, u32 cap, float* erow, float alpha,
                                             float& sq) {
     const u32 tk = (u32)(lo >> 32);
     const float thr = __uint_as_float(tk);
-    const u32 j0 = tile * (THREADS * UNROLL) + tid;
+    const u32 j0 = tile * (THREADS * UNROLL) + threadIdx.x;
     const uint4* p = g.vec + j0;
     uint4* pe = kEF ? reinterpret_cast<uint4*>(erow + g.head) + j0 : nullptr;
     uint4 v[UNROLL];
@@ -375,8 +373,8 @@ __device__ __forceinline__ void filter_tile(const RowGeom& g, u32 tile, u32 tid,
             }
         }
     }
-    if (tile == 0 && tid < 32 && (g.head | g.tail)) {
-        u32 lane = tid;
+    if (tile == 0 && threadIdx.x < 32 && (g.head | g.tail)) {
+        u32 lane = threadIdx.x;
         bool live = false;
         u32 idx = 0;
         if (lane < g.head) { live = true; idx = lane; }
@@ -404,27 +402,36 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
     extern __shared__ u64 sh_lo[];  // every row's bound, fetched once
     __shared__ uint2 sh_buf[(kFilterThreads / 32) * kStageSlots];
     __shared__ u32 sh_n[kFilterThreads / 32];
+    __shared__ u32 sh_claim[2];
     const u32 part = blockIdx.x / cpp;
-#if TK_FILTER_TRIGGER
-    allow_dependents();  // the kernel after this one takes the SMs as they fall free and waits there for this grid to end
-#endif
     if (part >= parts) return;
-    dependency_wait();  // the bounds come from the sampling kernel
+    dependency_wait();  // the bounds and the zeroed tickets come from the sampling kernel
     if (threadIdx.x == 0) phase_stamp(ctrl, kStampFilterStart);
     for (int r = threadIdx.x; r < rows; r += kFilterThreads) sh_lo[r] = rs[r].lo;
     if (threadIdx.x < kFilterThreads / 32) sh_n[threadIdx.x] = 0;
     __syncthreads();
     const WarpStage st = warp_stage(sh_buf, sh_n);
     const u64 total = (u64)rows * tpr;
-    const u64 t_end = (u64)(part + 1) * total / parts;
-    u64 t = (u64)part * total / parts + (blockIdx.x - part * cpp);
+    const u64 t_begin = (u64)part * total / parts, t_end = (u64)(part + 1) * total / parts;
+    // The last tiles of the range (about kFilterDynTiles per CTA, at most an eighth of the range) are
+    // not dealt out in advance but claimed one at a time from a counter: the CTAs of a range finish
+    // their fixed shares a few per cent apart (measured on the benchmark workload: 545 .. 572 us,
+    // no pattern from launch to launch), and with the claimed end they all run dry within a few
+    // tiles' time of each other.
+    // (not for short ranges, under 64 tiles per CTA: there the barrier per claimed tile costs more than the
+    // fixed shares differ)
+    u64 n_dyn = (u64)cpp * kFilterDynTiles;
+    if (n_dyn > (t_end - t_begin) / 8) n_dyn = (t_end - t_begin) / 8;
+    if ((t_end - t_begin) < (u64)cpp * 64) n_dyn = 0;
+    const u64 t_dyn = t_end - n_dyn;
+    u64 t = t_begin + (blockIdx.x - part * cpp);
     int cur = -1;
     RowGeom g;
     u64 lo = 0;
     int row = (int)(t / tpr);
     u32 tile = (u32)(t - (u64)row * tpr);
     float sq = 0.0f;
-    for (; t < t_end; t += cpp) {
+    for (; t < t_dyn; t += cpp) {
         if (row != cur) {
             if (cur >= 0) {
                 stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
@@ -435,11 +442,42 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
             lo = sh_lo[row];
         }
         if (tile * (u32)(kFilterThreads * kUnroll) < g.nv || tile == 0)
-            filter_tile<kFilterThreads, kUnroll, kEF, kStats>(g, tile, threadIdx.x, lo, st, rs + row, cand + (size_t)row * cap, cap,
+            filter_tile<kFilterThreads, kUnroll, kEF, kStats>(g, tile, lo, st, rs + row, cand + (size_t)row * cap, cap,
                                                               kEF ? ef.eps + (size_t)row * (size_t)d : nullptr, ef.alpha,
                                                               sq);
         tile += cpp;
         while (tile >= tpr) { tile -= tpr; ++row; }
+    }
+    if (n_dyn > 0) {
+        // sh_claim[i & 1] = the i-th claim of this CTA; the next one is asked for before the current tile
+        // is read and parked after it, so its round trip is hidden
+        u32* ticket = &rs[part].tile_ticket;  // zeroed by the sampling kernel (range numbers are row numbers too)
+        if (threadIdx.x == 0) sh_claim[0] = atomicAdd(ticket, 1u);
+        __syncthreads();
+        for (u32 i = 0;; ++i) {
+            const u32 c = sh_claim[i & 1];
+            if ((u64)c >= n_dyn) break;
+            u32 next_claim = 0;
+            if (threadIdx.x == 0) next_claim = atomicAdd(ticket, 1u);
+            t = t_dyn + c;
+            row = (int)(t / tpr);
+            tile = (u32)(t - (u64)row * tpr);
+            if (row != cur) {
+                if (cur >= 0) {
+                    stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
+                    if (kStats) { warp_add_double(&rs[cur].sum_sq, (double)sq); sq = 0.0f; }
+                }
+                cur = row;
+                g = row_geom(x, row, d);
+                lo = sh_lo[row];
+            }
+            if (tile * (u32)(kFilterThreads * kUnroll) < g.nv || tile == 0)
+                filter_tile<kFilterThreads, kUnroll, kEF, kStats>(g, tile, lo, st, rs + row, cand + (size_t)row * cap,
+                                                                  cap, kEF ? ef.eps + (size_t)row * (size_t)d : nullptr,
+                                                                  ef.alpha, sq);
+            if (threadIdx.x == 0) sh_claim[(i + 1) & 1] = next_claim;
+            __syncthreads();
+        }
     }
     if (cur >= 0) {
         stage_flush(st, rs + cur, cand + (size_t)cur * cap, cap);
@@ -522,31 +560,18 @@ __device__ __forceinline__ int build_row_list(int rows, unsigned short* sh_list,
     return (int)total;
 }
 
-// Shared memory of general_body (one CTA of kGeneralThreads threads).
-struct GeneralShared {
-    u32 hist[kHistBins];
-    unsigned short list[kMaxRowsPerLaunch];
-    u32 scratch[33];
-    u32 res[2];
-    uint2 buf[(kGeneralThreads / 32) * kStageSlots];
-    u32 n[kGeneralThreads / 32];
-};
-
-// Called by every thread of a cooperatively launched grid of kGeneralThreads-thread CTAs.
-// Returns without a grid-wide barrier when every row verified (all CTAs take the same branch:
-// they evaluate the same row states, which nothing modifies before the first barrier below —
-// a caller that goes on to select from the lists only adds to RowState.out_count / sel_sq,
-// which the vote does not read).
-__device__ __noinline__ void general_body(GeneralShared& sh, const float* __restrict__ x, int rows, int64_t d, u32 K,
-                                          u32 tpr, u32 cap, RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl,
-                                          int stats) {
-    u32* sh_hist = sh.hist;
-    unsigned short* sh_list = sh.list;
-    u32* sh_scratch = sh.scratch;
-    u32* sh_res = sh.res;
-    uint2* sh_buf = sh.buf;
-    u32* sh_n = sh.n;
+__global__ void __launch_bounds__(kGeneralThreads)
+general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr, u32 cap,
+               RowState* rs, u32* hist, uint2* cand, Ctrl* ctrl, int stats) {
+    __shared__ u32 sh_hist[kHistBins];
+    __shared__ unsigned short sh_list[kMaxRowsPerLaunch];
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_res[2];
+    __shared__ uint2 sh_buf[(kGeneralThreads / 32) * kStageSlots];
+    __shared__ u32 sh_n[kGeneralThreads / 32];
     cg::grid_group grid = cg::this_grid();
+    allow_dependents();  // the uplink select may queue up behind this grid
+    if (threadIdx.x == 0) phase_stamp(ctrl, kStampVerifyStart);
 
     // Which rows failed verification?  Nothing below modifies a RowState before
     // the first grid-wide barrier, so every CTA sees the same answer.
@@ -559,6 +584,7 @@ __device__ __noinline__ void general_body(GeneralShared& sh, const float* __rest
         for (int r = threadIdx.x; r < rows; r += blockDim.x) any |= failed(r) ? 1 : 0;
         if (!__syncthreads_or(any)) {
             if (blockIdx.x == 0 && threadIdx.x == 0) ctrl->rows_general = 0;
+            if (threadIdx.x == 0) phase_stamp(ctrl, kStampVerifyEnd);
             return;
         }
     }
@@ -682,12 +708,12 @@ __device__ __noinline__ void general_body(GeneralShared& sh, const float* __rest
         if ((u64)tile * kGeneralTileVecs >= (u64)g.nv && tile != 0) continue;
         {
             float unused = 0.0f;
-            filter_tile<kGeneralThreads, kStreamUnroll, false, false>(g, tile, threadIdx.x, lo, st, rs + row, cand + (size_t)row * cap,
+            filter_tile<kGeneralThreads, kStreamUnroll, false, false>(g, tile, lo, st, rs + row, cand + (size_t)row * cap,
                                                                       cap, nullptr, 0.0f, unused);
         }
     }
     if (cur >= 0) stage_flush(st, rs + row, cand + (size_t)row * cap, cap);
-    grid.sync();  // the redone rows' lists are complete before any CTA selects from them
+    if (threadIdx.x == 0) phase_stamp(ctrl, kStampVerifyEnd);
 }
 
 // ---------------------------------------------------------------------------
@@ -719,10 +745,6 @@ struct LinkArgs {
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
-#ifndef TK_GRID_PER_CTA
-#define TK_GRID_PER_CTA 4096
-#endif
-constexpr int kGridPerCta = TK_GRID_PER_CTA;  // grid-wide selection: list entries per CTA that holds any (0: spread over all CTAs)
 
 // Short rows with no sampled bound: the selection reads the row itself instead of a candidate
 // list (entry i is component i), which replaces the multi-pass kernel and its launches.
@@ -764,44 +786,37 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
 //   kGrid == true   a single row spread over the whole (cooperatively launched) grid, for
 //                   lists too long for one cluster (the union of N uplink messages);
 //                   histograms are combined in `ghist` (3 x kHistBins words of global
-//                   memory, all zero when the kernel starts), grid barriers between levels
+//                   memory, all zero when the kernel starts), grid barriers between levels.
+//                   With `prebuilt` the first level's histogram — every entry's key by its
+//                   leading 11 bits — is already complete in ghist[0 .. kHistBins) (the server
+//                   sum counted it while it appended the entries), so the first pass over the
+//                   list and its barrier are not needed.
 //
 // kDense (cluster variant only): the "list" of row r is the row dense.x[r][0..cap) itself, every
 // component a candidate; the kernel then also does what the sampling / reset kernels do for
 // the other paths (row state, union state).
-// Shared memory of select_body (one CTA of kSelectThreads threads).
-struct SelectShared {
-    u32 hist[2][kHistBins];  // double-buffered: peers may still read level L while L+1 fills
-    u32 tot[kHistBins];
-    u32 scratch[33];
-    u32 res[2];
-    u64 list[kRankMax];      // the bucket that gets ranked directly (cluster: gathered in CTA 0's copy)
-    u32 list_n;
-    u64 T;
-};
-
-// Selects row `row`.  Called by every thread of the row's cluster (kGrid == false) or of the whole
-// cooperatively launched grid (kGrid == true); a cluster may call it for one row after another.
-// prebuilt (grid variant): the first level's histogram — every entry's key by its leading 11 bits —
-// is already complete in ghist[0 .. kHistBins) (the server sum counted it while it appended the
-// entries), so the first pass over the list and its barrier are not needed.
-template <bool kGrid, bool kDense>
-__device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uint2* lists, size_t list_stride,
-                                            u32 cap, RowState* rs, u32 K, uint2* out, size_t out_stride,
-                                            const ApplyArgs& apply, const LinkArgs& link, Ctrl* ctrl, u32* ghist,
-                                            const DenseArgs& dense, bool prebuilt) {
-    u32 (*sh_hist)[kHistBins] = sh.hist;
-    u32* sh_tot = sh.tot;
-    u32* sh_scratch = sh.scratch;
-    u32* sh_res = sh.res;
-    u64* sh_list = sh.list;
-    u32& sh_list_n = sh.list_n;
-    u64& sh_T = sh.T;
+template <bool kGrid, bool kDense = false>
+__global__ void __launch_bounds__(kSelectThreads)
+select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowState* rs, u32 K,
+              uint2* out, size_t out_stride, ApplyArgs apply, LinkArgs link, Ctrl* ctrl, u32* ghist,
+              DenseArgs dense, int prebuilt) {
+    __shared__ u32 sh_hist[2][kHistBins];  // double-buffered: peers may still read level L while L+1 fills
+    __shared__ u32 sh_tot[kHistBins];
+    __shared__ u32 sh_scratch[33];
+    __shared__ u32 sh_res[2];
+    __shared__ u64 sh_list[kRankMax];  // the bucket that gets ranked directly (cluster: gathered in CTA 0's copy)
+    __shared__ u32 sh_list_n;
+    __shared__ u64 sh_T;
     cg::cluster_group cluster = cg::this_cluster();
     cg::grid_group grid = cg::this_grid();
     if (threadIdx.x == 0) sh_list_n = 0;  // read by peers only after a cluster barrier
+    dependency_wait();   // candidates and bounds come from the kernels before
+    allow_dependents();
+    constexpr int stamp0 = kGrid ? kStampDownStart : kStampUpStart;  // start, loaded, level, threshold, end
+    if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0);
     const u32 CS = kGrid ? gridDim.x : cluster.num_blocks();
     const u32 rank = kGrid ? blockIdx.x : cluster.block_rank();
+    const u32 row = kGrid ? 0u : blockIdx.x / CS;
     RowState* r = rs + row;
     if (kDense) {
         if (rank == 0 && threadIdx.x == 0) {
@@ -819,16 +834,10 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
     const uint2* list = kDense ? nullptr : lists + (size_t)row * list_stride;
     const float* xrow = kDense ? dense.x + (size_t)row * list_stride : nullptr;
     auto read_entry = [&](u32 i) -> uint2 {
-        // lists may have been written earlier in the same launch (redone rows, the union): L2, not the read-only path
-        return kDense ? make_uint2(i, __float_as_uint(__ldg(xrow + i))) : __ldcg(&list[i]);
+        return kDense ? make_uint2(i, __float_as_uint(__ldg(xrow + i))) : list[i];
     };
-    // Grid variant: every CTA takes part in the barriers and reads the combined histograms, but the
-    // entries are dealt to the first CSd CTAs only (about kGridPerCta each): fewer CTAs push their
-    // counts into the global histogram.  The others hold nothing (base = C: every index test fails).
-    const u32 CSd = (kGrid && kGridPerCta > 0) ? min(CS, max(1u, (C + (u32)kGridPerCta - 1u) / (u32)kGridPerCta)) : CS;
-    const u32 base = rank < CSd ? rank * kSelectThreads : C;
-    const u32 first = base + threadIdx.x;
-    const u32 stride = CSd * kSelectThreads;
+    const u32 first = rank * kSelectThreads + threadIdx.x;
+    const u32 stride = CS * kSelectThreads;
     const u32 rest = first + kSelectRegs * stride;  // entries from here on are re-read every level
 
     // this thread's entries first + k*stride, k < kSelectRegs, stay in registers as composite
@@ -863,17 +872,17 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
         warp_add_double(&r->sum_sq, (double)sq);
     }
 
-    const int stamp0 = kGrid ? kStampDownLoaded : kStampUpLoaded;
-    if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0);
+    if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 1);
     u64 T = 1;  // emit entries with ck >= T (absent ones are 0)
-    const bool solo = kGrid && CS == 1 && !prebuilt;  // one CTA and nothing to fetch from the global scratch
-    if (kGrid && prebuilt && C <= Keff && rank == 0)  // nothing to select: the prebuilt counts are not needed
+    const bool pre = kGrid && prebuilt != 0;
+    const bool solo = kGrid && CS == 1 && !pre;  // one CTA and nothing to fetch from the global scratch
+    if (pre && C <= Keff && rank == 0)  // nothing to select: the prebuilt counts are not needed
         for (int b = threadIdx.x; b < kHistBins; b += kSelectThreads) ghist[b] = 0;
     if (C > Keff) {
         u64 lo = max(r->lo, 1ull);
         u64 hi = kDense ? 0x7fffffffffffffffull : ((u64)r->max_key << 32) | 0xffffffffull;  // dense: no maximum is known
-        if (kGrid && prebuilt) {  // the whole range: 2048 buckets of 2^52 composite keys = keys by their leading 11 bits
-            lo = 1ull;            // (ck - 1) >> 52 == key >> 20 for every real entry: its index bits are never all zero)
+        if (pre) {      // the whole range: 2048 buckets of 2^52 composite keys = keys by their leading 11 bits
+            lo = 1ull;  // ((ck - 1) >> 52 == key >> 20 for every real entry: its index bits are never all zero)
             hi = 0x7fffffffffffffffull;
         }
         if (hi < lo) hi = lo;
@@ -884,7 +893,7 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
             u64 width = hi - lo;
             int s = width ? max(0, 64 - __clzll((long long)width) - 11) : 0;
             int nb = (int)(width >> s) + 1;
-            const bool ready = kGrid && prebuilt && level == 0;  // this level's counts are already in ghist
+            const bool ready = pre && level == 0;  // this level's counts are already in ghist
             if (threadIdx.x == 0) sh_res[0] = 0xffffffffu;
             if (!ready) {
                 for (int b = threadIdx.x; b < nb; b += kSelectThreads) hist[b] = 0;
@@ -934,7 +943,7 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
                 if (threadIdx.x == 0 && rank == 0) raise_status(ctrl, -5);
                 break;
             }
-            if (TK_PHASE_CLOCK && !kDense && level == 0 && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 1);
+            if (TK_PHASE_CLOCK && !kDense && level == 0 && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 2);
             need -= above;
             u64 blo = lo + ((u64)b << s);
             u64 bhi = blo + ((1ull << s) - 1ull);
@@ -1012,7 +1021,7 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
         }
     }
 
-    if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 2);
+    if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 3);
     // emission: every entry with ck >= T, exactly Keff of them; one counter update per warp
     uint2* orow = out + (size_t)row * out_stride;
     double sel_sq = 0.0;
@@ -1037,7 +1046,6 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
             base = __shfl_sync(0xffffffffu, base, 31);
         }
         const u32 slot0 = base + incl - mine;
-        if (TK_PHASE_CLOCK && !kGrid && !kDense && threadIdx.x == 0) phase_stamp(ctrl, kStampUpSlots);
         // The entries of one thread go to different coordinates, so their memory round trips (the
         // old value of w, the previous head of the chain) are independent: issue them all, then
         // finish them all, instead of one dependent load-store pair after the other.
@@ -1058,13 +1066,6 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
                 }
                 ++slot;
             }
-        }
-        if (TK_PHASE_CLOCK && !kGrid && !kDense) {
-            u32 any = 0;
-#pragma unroll
-            for (int k = 0; k < kSelectRegs; ++k) any |= fetched[k];
-            if (__syncthreads_or(any == 0xdeadbeefu)) raise_status(ctrl, -5);  // waits for every answer
-            if (threadIdx.x == 0) phase_stamp(ctrl, kStampUpFetched);
         }
         slot = slot0;
 #pragma unroll
@@ -1092,7 +1093,7 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
             }
         }
     }
-    for (u32 i0 = base + kSelectRegs * stride; i0 < C; i0 += stride) {
+    for (u32 i0 = rank * kSelectThreads + kSelectRegs * stride; i0 < C; i0 += stride) {
         u32 i = i0 + threadIdx.x;
         bool pred = false;
         uint2 e = make_uint2(0, 0);
@@ -1113,17 +1114,10 @@ __device__ __forceinline__ void select_body(SelectShared& sh, u32 row, const uin
         }
     }
     if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
-}
-
-// Few short rows: one cluster per row selects straight from the row (no lists, no bound).
-__global__ void __launch_bounds__(kSelectThreads)
-select_dense_kernel(size_t row_stride, u32 d, RowState* rs, u32 K, uint2* out, ApplyArgs apply, LinkArgs link, Ctrl* ctrl,
-                    DenseArgs dense) {
-    __shared__ SelectShared sh;
-    dependency_wait();
-    allow_dependents();
-    select_body<false, true>(sh, blockIdx.x / cg::this_cluster().num_blocks(), nullptr, row_stride, d, rs, K, out, (size_t)K,
-                             apply, link, ctrl, nullptr, dense, false);
+    if (TK_PHASE_CLOCK && !kDense) {
+        __syncthreads();
+        if (threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 4);
+    }
 }
 
 }  // namespace tk
