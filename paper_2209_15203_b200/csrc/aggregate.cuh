@@ -40,12 +40,21 @@ constexpr int kSlotWorkers = 128;  // the slot table is used up to this many wor
 // selection's emission does on the fly when the messages are produced on this GPU.
 // Also resets the union's state for the step.
 __global__ void __launch_bounds__(256)
-agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, u32* head, u32* next, u32* slots, u32 row_words,
-                RowState* uni, Ctrl* ctrl, u32 d) {
+agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p, u32* head, u32* next,
+                u32* slots, u32 row_words, RowState* uni, Ctrl* ctrl, u32 d) {
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) {
         uni->lo = 0; uni->cand_count = 0; uni->max_key = 0; uni->out_count = 0; uni->flags = 0;
         uni->sum_sq = 0.0; uni->sel_sq = 0.0; uni->nnz = 0;
+    }
+    // the downlink selection's first level wants a key no single worker's term lies below (union_bin):
+    // here, with no row thresholds at hand, the smallest p_q * |v| itself (bin_base was set to the
+    // largest value when the messages were produced, see reset_state)
+    {
+        u32 k = 0xffffffffu;
+        if (e < total) k = key_of(__float_as_uint(__fmul_rn(p[e / K_up], __uint_as_float(up[e].y))));
+        k = __reduce_min_sync(0xffffffffu, k);
+        if (lane_id() == 0 && k != 0xffffffffu) atomicMin(&uni->bin_base, k);
     }
     if (e >= total) return;
     u32 j = up[e].x;
@@ -66,13 +75,13 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,
                   int stats, u32* level0) {
     // level0, when given (kHistBins words of global memory, zero on entry): the sums' keys are also
-    // counted by their leading 11 bits — the first level of the downlink selection, complete when
-    // this grid ends
+    // counted by union_bin — the first level of the downlink selection, complete when this grid ends
     __shared__ u32 sh_hist[kHistBins];
     if (level0)
         for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
     dependency_wait();   // the entries are filed by the kernel before
     if (threadIdx.x == 0) phase_stamp(ctrl, kStampAggStart);
+    const u32 bin_base = level0 ? union_base(uni) : 0u;
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;
     u32 j = 0, own_bits = 0;
@@ -191,7 +200,7 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
     if (level0) {
         // the sums crowd into a few bins: one shared-memory atomic per distinct bin and warp
         // (the scan above has passed a barrier since sh_hist was cleared)
-        const u32 bin = key_of(bits) >> 20;
+        const u32 bin = union_bin(key_of(bits), bin_base);
         const u32 peers = __match_any_sync(0xffffffffu, owner ? bin : 0xffffffffu);
         if (owner && (int)lane_id() == __ffs(peers) - 1) atomicAdd(&sh_hist[bin], (u32)__popc(peers));
     } else if (ucap <= 4096u) {

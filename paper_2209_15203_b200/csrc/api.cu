@@ -393,6 +393,9 @@ int cluster_size_for(int64_t entries, int64_t rows, int sms) {
 #ifndef TK_PDL
 #define TK_PDL 1
 #endif
+#ifndef TK_COOP_PDL
+#define TK_COOP_PDL 1
+#endif
 
 // Launch with the programmatic-serialization attribute (the kernel calls dependency_wait()) and,
 // optionally, a cluster size.
@@ -599,11 +602,31 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             u64 gtiles = (u64)nr * b.tpr_general;
             unsigned ggrid = (unsigned)(gtiles < (u64)di->general_grid ? gtiles : (u64)di->general_grid);
             if (ggrid < 1) ggrid = 1;
+#if TK_COOP_PDL
+            {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(ggrid);
+                cfg.blockDim = dim3(kGeneralThreads);
+                cfg.stream = stream;
+                cudaLaunchAttribute attr[2];
+                attr[0].id = cudaLaunchAttributeCooperative;
+                attr[0].val.cooperative = 1;
+                attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[1].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 2;
+                if (cudaLaunchKernelExC(&cfg, (const void*)general_kernel, args) != cudaSuccess) {
+                    cudaGetLastError();
+                    return TK_ERR_CUDA;
+                }
+            }
+#else
             if (cudaLaunchCooperativeKernel((void*)general_kernel, dim3(ggrid), dim3(kGeneralThreads), args,
                                             0, stream) != cudaSuccess) {
                 cudaGetLastError();
                 return TK_ERR_CUDA;
             }
+#endif
             if (!predict && ev1 && r0 == 0) cudaEventRecord(ev1, stream);
             *launches += 1;
         }
@@ -911,7 +934,8 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
                         nullptr, &c->launches);
         if (rc != TK_OK) return rc;
     }
-    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0, c->slots, c->slot_row_words};
+    LinkArgs link = {c->head, c->next, (u32)c->d, 0, with_ef ? c->eps : nullptr, (size_t)c->d, 0, c->slots, c->slot_row_words,
+                     c->p, c->uni};
     EfArgs ef = {with_ef ? c->eps : nullptr, alpha};
     SelectBufs up = c->up;
     if (c->cand_cap > 0) up.cap = capped(up.cap, c->cand_cap, c->K_up);  // shorter lists, packed closer in the same buffer
@@ -952,8 +976,9 @@ int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_
     float* eps = with_ef ? c->eps + (size_t)row0 * (size_t)c->d : nullptr;
     LinkArgs link = {nullptr, nullptr, 0, 0, eps, (size_t)c->d, 0};  // chains are built after the exchange
     EfArgs ef = {eps, alpha};
+    // (the union's state is reset here too: the filing kernel of tk_step_server lowers its bin_base)
     return run_select(c->stream, grads_local_dev, rows, c->d, c->K_up, b, c->ctrl, c->force_general != 0, nullptr,
-                      nullptr, &c->launches, nullptr, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0);
+                      nullptr, &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0);
 }
 
 int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {
@@ -966,7 +991,7 @@ int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {
 int tk_step_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     if (!step_args_ok(c, alpha, mode) || !aligned4(w_dev)) return TK_ERR_INVALID;
     u32 total = (u32)(c->N * c->K_up);
-    agg_link_kernel<<<(total + 255) / 256, 256, 0, c->stream>>>(c->up.out, total, (u32)c->K_up, c->head, c->next, c->slots,
+    agg_link_kernel<<<(total + 255) / 256, 256, 0, c->stream>>>(c->up.out, total, (u32)c->K_up, c->p, c->head, c->next, c->slots,
                                                                  c->slot_row_words, c->uni, c->ctrl, (u32)c->d);
     TK_LAUNCH_CHECK();
     c->launches += 1;

@@ -91,6 +91,8 @@ struct RowState {
     double sel_sq;   // sum of squares of the emitted entries
     u32 nnz;         // union list: entries whose value is not zero
     u32 tile_ticket; // streaming pass: tiles handed out so far from the claimed end of tile range number <this row's index>
+    u32 bin_base;    // union: a key no unshared sum of this step lies below (see union_base)
+    u32 bin_hint;    // union: where the previous step's downlink threshold puts the buckets (0: none yet); survives resets
 };
 
 // Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the
@@ -131,6 +133,29 @@ __device__ __forceinline__ void phase_stamp(Ctrl* ctrl, int which) {
 }
 
 __device__ __forceinline__ u32 key_of(u32 bits) { return bits & 0x7fffffffu; }
+
+// First level of the downlink selection, counted by the server sum as it appends the union:
+// bucket 0 holds the keys below `base`, buckets 1 .. 2046 are 2^kUnionBinShift keys wide from
+// `base` on, bucket 2047 everything above.  Where the buckets sit is only a matter of speed (the
+// selection refines whatever bucket the K-th largest falls in): they are centred on the previous
+// step's threshold (bin_hint: +-24 % in value, 0.02 % per bucket — consecutive steps of a
+// training run have close thresholds, and then the bucket of the K-th holds few enough entries to
+// be ranked directly); without one they start at the smallest p_q * |K-th value of row q|, below
+// which no sum of a coordinate that only one worker sent can lie.
+#ifndef TK_UNION_BIN_SHIFT
+#define TK_UNION_BIN_SHIFT 11
+#endif
+constexpr int kUnionBinShift = TK_UNION_BIN_SHIFT;
+__device__ __forceinline__ u32 union_base(const RowState* uni) { return uni->bin_hint ? uni->bin_hint : uni->bin_base; }
+__device__ __forceinline__ u32 union_hint(u32 threshold_key) {  // the threshold in the middle bucket
+    const u32 half = (u32)(kHistBins / 2 - 1) << kUnionBinShift;
+    return threshold_key > half ? threshold_key - half : 1u;
+}
+__device__ __forceinline__ u32 union_bin(u32 key, u32 base) {
+    if (key < base) return 0u;
+    const u32 b = 1u + ((key - base) >> kUnionBinShift);
+    return b > (u32)(kHistBins - 1) ? (u32)(kHistBins - 1) : b;
+}
 
 __device__ __forceinline__ u64 composite(u32 key, u32 idx) {
     return ((u64)key << 32) | (u64)(0xffffffffu - idx);

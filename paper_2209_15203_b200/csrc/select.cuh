@@ -48,6 +48,7 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->flags = flags;
     r->ticket = 0;
     r->tile_ticket = 0;
+    r->bin_base = 0xffffffffu;
     r->g_active = 0;
     r->sum_sq = 0.0;
     r->sel_sq = 0.0;
@@ -204,6 +205,9 @@ __device__ __forceinline__ RowGeom row_geom(const float* x, int row, int64_t d) 
 // Candidates are first collected per warp in shared memory and appended to the
 // row's list in batches: hits cluster in the layers with the largest scale, and
 // one global atomic per hit on the row's single counter would serialise there.
+#ifndef TK_COOP_PDL
+#define TK_COOP_PDL 1
+#endif
 #ifndef TK_STAGE_SLOTS
 #define TK_STAGE_SLOTS 128
 #endif
@@ -404,6 +408,9 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
     __shared__ u32 sh_n[kFilterThreads / 32];
     __shared__ u32 sh_claim[2];
     const u32 part = blockIdx.x / cpp;
+#if TK_COOP_PDL
+    allow_dependents();
+#endif
     if (part >= parts) return;
     dependency_wait();  // the bounds and the zeroed tickets come from the sampling kernel
     if (threadIdx.x == 0) phase_stamp(ctrl, kStampFilterStart);
@@ -571,6 +578,7 @@ general_kernel(const float* __restrict__ x, int rows, int64_t d, u32 K, u32 tpr,
     __shared__ u32 sh_n[kGeneralThreads / 32];
     cg::grid_group grid = cg::this_grid();
     allow_dependents();  // the uplink select may queue up behind this grid
+    dependency_wait();   // (returns at once unless launched as a programmatic dependent)
     if (threadIdx.x == 0) phase_stamp(ctrl, kStampVerifyStart);
 
     // Which rows failed verification?  Nothing below modifies a RowState before
@@ -742,6 +750,10 @@ struct LinkArgs {
     // of the slot table (row_words words per row, all zero at rest); see aggregate.cuh.
     u32* slots;
     u32 row_words;
+    // server step, for the downlink selection's first level (union_bin): the weights p_q and the
+    // union's state, whose bin_base every row lowers to p_q * |its K-th value|
+    const float* p;
+    RowState* uni;
 };
 
 constexpr int kSelectRegs = 12;  // entries each thread keeps in registers across the levels
@@ -787,10 +799,10 @@ __device__ __forceinline__ void emit_entry(u32 row, u32 slot, u32 Keff, u32 idx,
 //                   lists too long for one cluster (the union of N uplink messages);
 //                   histograms are combined in `ghist` (3 x kHistBins words of global
 //                   memory, all zero when the kernel starts), grid barriers between levels.
-//                   With `prebuilt` the first level's histogram — every entry's key by its
-//                   leading 11 bits — is already complete in ghist[0 .. kHistBins) (the server
-//                   sum counted it while it appended the entries), so the first pass over the
-//                   list and its barrier are not needed.
+//                   With `prebuilt` the first level's histogram — every entry's key by
+//                   union_bin — is already complete in ghist[0 .. kHistBins) (the server sum
+//                   counted it while it appended the entries), so the first pass over the list
+//                   and its barrier are not needed.
 //
 // kDense (cluster variant only): the "list" of row r is the row dense.x[r][0..cap) itself, every
 // component a candidate; the kernel then also does what the sampling / reset kernels do for
@@ -881,8 +893,8 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     if (C > Keff) {
         u64 lo = max(r->lo, 1ull);
         u64 hi = kDense ? 0x7fffffffffffffffull : ((u64)r->max_key << 32) | 0xffffffffull;  // dense: no maximum is known
-        if (pre) {      // the whole range: 2048 buckets of 2^52 composite keys = keys by their leading 11 bits
-            lo = 1ull;  // ((ck - 1) >> 52 == key >> 20 for every real entry: its index bits are never all zero)
+        if (pre) {  // the whole range; the first level's buckets are union_bin's, all kHistBins of them
+            lo = 1ull;
             hi = 0x7fffffffffffffffull;
         }
         if (hi < lo) hi = lo;
@@ -948,6 +960,14 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
             u64 blo = lo + ((u64)b << s);
             u64 bhi = blo + ((1ull << s) - 1ull);
             if (bhi > hi) bhi = hi;
+            if (ready) {  // bucket b of union_bin as a range of composite keys
+                const u64 base = union_base(r);
+                const u64 klo = b == 0u ? 0ull : base + ((u64)(b - 1u) << kUnionBinShift);
+                u64 khi = b == 0u ? base - 1ull : klo + ((1ull << kUnionBinShift) - 1ull);  // (bucket 0 is empty when base is 0)
+                if (b == (u32)(kHistBins - 1) || khi > 0x7fffffffull) khi = 0x7fffffffull;
+                blo = max(klo << 32, 1ull);
+                bhi = (khi << 32) | 0xffffffffull;
+            }
             const u32 cnt = sh_tot[b];
             lo = blo;
             hi = bhi;
@@ -1022,6 +1042,11 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
     }
 
     if (TK_PHASE_CLOCK && !kDense && threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 3);
+    if (!kGrid && link.uni && rank == 0 && threadIdx.x == 0) {
+        // no emitted magnitude of this row is below its K-th value (key T >> 32; 0 when the whole list goes out)
+        const float least = __fmul_rn(link.p[link.row_base + row], __uint_as_float((u32)(T >> 32)));
+        atomicMin(&link.uni->bin_base, key_of(__float_as_uint(least)));
+    }
     // emission: every entry with ck >= T, exactly Keff of them; one counter update per warp
     uint2* orow = out + (size_t)row * out_stride;
     double sel_sq = 0.0;
@@ -1114,6 +1139,9 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         }
     }
     if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
+    // the next step's first level is centred on this step's threshold (every CTA is past its last look
+    // at the buckets: a grid barrier lies behind whenever they were used)
+    if (kGrid && prebuilt && rank == 0 && threadIdx.x == 0) r->bin_hint = C > Keff ? union_hint((u32)(T >> 32)) : 0u;
     if (TK_PHASE_CLOCK && !kDense) {
         __syncthreads();
         if (threadIdx.x == 0) phase_stamp(ctrl, stamp0 + 4);
