@@ -230,6 +230,8 @@ def main():
     ap.add_argument("--agree", type=float, default=None, metavar="C",
                     help="workers see noisy copies of one shared vector, row_q = base * (1 + C z_q), instead of "
                          "independent rows: their selections then mostly coincide (union near K)")
+    ap.add_argument("--no-bound-reuse", action="store_true", help="sample every row's bound in every step instead of "
+                    "keeping the bounds that served the step before (tk_set_bound_reuse)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -275,6 +277,8 @@ def main():
         ctx.tk_ef_attach()
     if args.force_general:
         ctx.tk_set_force_general(True)
+    if args.no_bound_reuse:
+        ctx.tk_set_bound_reuse(False)
 
     def barrier():
         replicas.barrier()
@@ -397,7 +401,10 @@ def main():
                     "launch": ("CUDA graph replay; every %d-th step plain launches with timestamps around the "
                                "streaming kernel" % max(1, args.profile_every)) if args.graph else "stream launches",
                     "parallelism": ("workers sharded over %d ranks, one all-gather per step" if args.sharded
-                                    else "replicas x%d") % world})
+                                    else "replicas x%d") % world,
+                    "bounds": "sampled in every step" if args.no_bound_reuse else
+                              "kept from the step before where they admitted 1.25 K .. 4 K candidates (verified "
+                              "exactly every step), sampled otherwise; --no-bound-reuse samples every step"})
         if args.agree is not None:
             cfg["rows"] = "shared vector x (1 + %g z_q)" % args.agree
         cfg["input_checksum_step0"] = "%016x" % sum_checksum(bufs[0])

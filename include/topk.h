@@ -348,6 +348,19 @@ int tk_set_force_general(tk_ctx* ctx, int on);
  */
 int tk_set_cand_cap(tk_ctx* ctx, int64_t cap);
 
+/*
+ * Bound reuse (on by default; no counterpart in the paper, which says nothing about how Top_K is
+ * computed).  The uplink selection of a long row first needs a lower bound of the row's K-th
+ * magnitude; normally it is estimated from a sample of the row at the start of every step.  With
+ * reuse on, a row whose bound admitted between 1.25 K and 4 K candidates in the context's last
+ * step keeps that bound for the next step and skips the sampling — consecutive iterations of a
+ * training run have close thresholds.  Results are identical either way (every bound is verified
+ * by the exact count of the components it admits, and a row whose bound fails is redone exactly
+ * in the same step); only the time differs: a step whose vectors differ a lot in scale from the
+ * step before pays one multi-pass redo.  tk_set_bound_reuse(ctx, 0) samples every step.
+ */
+int tk_set_bound_reuse(tk_ctx* ctx, int on);
+
 /* Kernels launched on the context's stream since tk_init. */
 int64_t tk_launch_count(tk_ctx* ctx);
 

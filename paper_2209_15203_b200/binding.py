@@ -23,7 +23,7 @@ TK_MODE_EF = 2
 EXPORTS = ["tk_workspace_bytes", "tk_init", "tk_step", "tk_step_uplink", "tk_messages", "tk_step_server", "tk_step_host", "tk_topk", "tk_topk_noalloc", "tk_topk_noalloc_status", "tk_ef_bytes",
            "tk_ef_attach", "tk_ef_state", "tk_set_diagnostics", "tk_diagnostics", "tk_set_kdown",
            "tk_last_uplink", "tk_last_aggregate", "tk_last_downlink", "tk_status", "tk_set_profile",
-           "tk_set_force_general", "tk_set_cand_cap", "tk_comm_model", "tk_set_graph", "tk_launch_count", "tk_debug_phase_clock", "tk_destroy", "tk_release_scratch", "tk_strerror"]
+           "tk_set_force_general", "tk_set_cand_cap", "tk_set_bound_reuse", "tk_comm_model", "tk_set_graph", "tk_launch_count", "tk_debug_phase_clock", "tk_destroy", "tk_release_scratch", "tk_strerror"]
 
 
 class TkError(RuntimeError):
@@ -90,6 +90,8 @@ def load(build_if_missing: bool = True):
     lib.tk_topk_noalloc.restype = ctypes.c_int
     lib.tk_topk_noalloc_status.argtypes = []
     lib.tk_topk_noalloc_status.restype = ctypes.c_int
+    lib.tk_set_bound_reuse.argtypes = [vp, ctypes.c_int]
+    lib.tk_set_bound_reuse.restype = ctypes.c_int
     lib.tk_set_cand_cap.argtypes = [vp, i64]
     lib.tk_set_cand_cap.restype = ctypes.c_int
     lib.tk_comm_model.argtypes = [i32, i64, i64, i64, ctypes.c_double, ctypes.c_double, ctypes.c_double,
@@ -291,6 +293,9 @@ class Context:
 
     def tk_set_force_general(self, on: bool) -> None:
         _check(load().tk_set_force_general(self._h, 1 if on else 0), "tk_set_force_general")
+
+    def tk_set_bound_reuse(self, on: bool) -> None:
+        _check(load().tk_set_bound_reuse(self._h, 1 if on else 0), "tk_set_bound_reuse")
 
     def tk_set_cand_cap(self, cap: int) -> None:
         """Testing aid: cap every row's candidate list (0 restores the laid-out capacity)."""

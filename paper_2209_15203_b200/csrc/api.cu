@@ -278,6 +278,7 @@ struct tk_ctx {
     u32 ucap = 0;
     // host state
     int force_general = 0;
+    int bound_reuse = 1;       // tk_set_bound_reuse
     int64_t cand_cap = 0;      // tk_set_cand_cap: 0 = the capacity the workspace was laid out for
     int diagnostics = 0;
     int profile = 0;           // 0 = off, n = timestamp the streaming pass of every n-th step
@@ -492,7 +493,8 @@ int launch_select_grid(cudaStream_t stream, int ctas, const uint2* list, u32 cap
 int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int64_t K, const SelectBufs& b,
                Ctrl* ctrl, bool force_general, cudaEvent_t ev0, cudaEvent_t ev1, int64_t* launches,
                RowState* also_reset = nullptr, LinkArgs link = LinkArgs{nullptr, nullptr, 0, 0},
-               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}, bool stats = false) {
+               EfArgs ef = EfArgs{nullptr, 0.0f}, ApplyArgs apply = ApplyArgs{nullptr, 0.0f}, bool stats = false,
+               bool reuse = false /* rows may keep the bound of their last selection (predict_kernel) */) {
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
@@ -536,13 +538,13 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             const bool light = turns <= (fused ? kPredictLightTurns / 2 : kPredictLightTurns);
             dim3 pg(kPredictCtas, nr);
             if (fused && light)
-                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl);
+                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
             else if (fused)
-                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl);
+                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
             else if (light)
-                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl);
+                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
             else
-                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl);
+                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             u32 tprf = fused ? b.tpr_filter_ef : b.tpr_filter;
@@ -940,7 +942,7 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
     SelectBufs up = c->up;
     if (c->cand_cap > 0) up.cap = capped(up.cap, c->cand_cap, c->K_up);  // shorter lists, packed closer in the same buffer
     rc = run_select(s, grads_dev, c->N, c->d, c->K_up, up, c->ctrl, c->force_general != 0, e0, e1,
-                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag);
+                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag, c->bound_reuse != 0);
     if (rc != TK_OK) return rc;
     rc = run_server(c, w_dev, alpha, mode);
     if (rc != TK_OK || !gap) return rc;
@@ -978,7 +980,8 @@ int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_
     EfArgs ef = {eps, alpha};
     // (the union's state is reset here too: the filing kernel of tk_step_server lowers its bin_base)
     return run_select(c->stream, grads_local_dev, rows, c->d, c->K_up, b, c->ctrl, c->force_general != 0, nullptr,
-                      nullptr, &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0);
+                      nullptr, &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0,
+                      c->bound_reuse != 0);
 }
 
 int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {
@@ -1317,6 +1320,13 @@ int tk_set_graph(tk_ctx* c, int on) {
 int tk_set_force_general(tk_ctx* c, int on) {
     if (!c) return TK_ERR_INVALID;
     c->force_general = on ? 1 : 0;
+    return TK_OK;
+}
+
+int tk_set_bound_reuse(tk_ctx* c, int on) {
+    if (!c) return TK_ERR_INVALID;
+    if ((on != 0) != (c->bound_reuse != 0)) drop_graphs(c);  // captured steps carry the old setting
+    c->bound_reuse = on ? 1 : 0;
     return TK_OK;
 }
 

@@ -93,6 +93,8 @@ struct RowState {
     u32 tile_ticket; // streaming pass: tiles handed out so far from the claimed end of tile range number <this row's index>
     u32 bin_base;    // union: a key no unshared sum of this step lies below (see union_base)
     u32 bin_hint;    // union: where the previous step's downlink threshold puts the buckets (0: none yet); survives resets
+    u32 reuse_ok;    // the bound `lo` served the last selection well and may serve the next one (see predict_kernel); survives resets
+    u32 pad_;
 };
 
 // Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the

@@ -40,6 +40,14 @@ namespace tk {
 // lower bound of the `rank`-th largest maximum — exact in its leading 22 bits,
 // which costs two histogram passes instead of four — as the row's bound: at
 // least `rank` sampled values are >= it.
+//
+// Bound reuse.  Consecutive steps of a training run have close thresholds, so a bound that
+// admitted a comfortable number of candidates in the last selection of this row (between 1.25 K
+// and 4 K, all verified; RowState.reuse_ok, set by the selection kernel) is simply kept when
+// `reuse` is set: the row's CTAs return at once, no sample is read and nothing is ranked.  The
+// result stays exact either way — the bound is verified by the exact count as always, and a row
+// whose count leaves the window is sampled again in the step after (a row whose count falls
+// below K or above the list's capacity is redone by the multi-pass path in the same step).
 __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->lo = lo;
     r->cand_count = 0;
@@ -60,7 +68,7 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
 template <bool kEF, bool kLight>
 __global__ void __launch_bounds__(kPredictThreads, kLight ? 2 : 1)
 predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank, u32 K,
-               RowState* rs, u32* smax, RowState* also_reset, EfArgs ef, Ctrl* ctrl) {
+               RowState* rs, u32* smax, RowState* also_reset, EfArgs ef, Ctrl* ctrl, int reuse) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
@@ -70,6 +78,13 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     const int row = blockIdx.y;
     const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;   // 0 .. 2*kSampleSlots-1
     if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
+    if (reuse && rs[row].reuse_ok) {  // the same answer in all CTAs of the row: nothing here writes reuse_ok
+        if (t == 0) {
+            reset_state(rs + row, rs[row].lo, 0u);
+            phase_stamp(ctrl, kStampPredictEnd);
+        }
+        return;
+    }
     const float* xr = x + (size_t)row * (size_t)d;
     const float* er = kEF ? ef.eps + (size_t)row * (size_t)d : nullptr;
     // runs start at multiples of 32 elements
@@ -1139,6 +1154,12 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         }
     }
     if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
+    // may the row's bound serve the next selection too?  (cand_count is not written by this kernel)
+    if (!kGrid && !kDense && rank == 0 && threadIdx.x == 0) {
+        const u64 cc = r->cand_count;
+        r->reuse_ok = ((r->flags & kRowGeneral) == 0u && (u32)r->lo == 0u && r->lo != 0ull && cc * 4u >= (u64)K * 5u &&
+                       cc <= (u64)K * 4u && cc <= (u64)cap) ? 1u : 0u;
+    }
     // the next step's first level is centred on this step's threshold (every CTA is past its last look
     // at the buckets: a grid barrier lies behind whenever they were used)
     if (kGrid && prebuilt && rank == 0 && threadIdx.x == 0) r->bin_hint = C > Keff ? union_hint((u32)(T >> 32)) : 0u;

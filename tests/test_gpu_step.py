@@ -132,6 +132,32 @@ def test_forced_list_overflow_redoes_every_row_exactly():
         ctx.close()
 
 
+def test_kept_bounds_survive_changes_of_scale():
+    # A row keeps the bound of the step before when that bound admitted a comfortable number of
+    # candidates (tk_set_bound_reuse, on by default).  Steps of the same distribution then take the
+    # single streaming pass without sampling; a step whose vectors are a thousand times smaller (the
+    # kept bound admits nothing) or larger (it admits everything, the lists overflow) must be redone
+    # by the exact multi-pass path, and the step after that samples afresh.  Results are the oracle's
+    # throughout; with reuse off no step needs the multi-pass path.
+    wl = W.workload(2, d=700_003, N=5)
+    scales = (1.0, 1.0, 1e-3, 1.0, 1.0, 1e3, 1.0, 0.97, 1.04)
+    for reuse in (True, False):
+        ctx = make_ctx(wl, wl.K_down[0])
+        ctx.tk_set_bound_reuse(reuse)
+        w_dev = W.make_w(wl, DEV)
+        w_ref = w_dev.cpu().numpy()
+        general = []
+        for s, c in enumerate(scales):
+            G = W.make_grads(wl, s, DEV) * c
+            w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, 1, wl.K_down[0], "scale %g reuse=%s" % (c, reuse))
+            general.append(ctx.tk_status().rows_general)
+        if reuse:
+            assert general == [0, 0, wl.N, 0, 0, wl.N, 0, 0, 0], general
+        else:
+            assert general == [0] * len(scales), general
+        ctx.close()
+
+
 def test_kdown_larger_than_union_pads_with_zero_entries():
     wl = W.workload(4, d=400_000, N=4)          # K_up = 40, union <= 160; K_down = 4000 > |U|
     assert wl.K_down[-1] > wl.N * wl.K_up
