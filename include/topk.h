@@ -357,7 +357,8 @@ int tk_set_cand_cap(tk_ctx* ctx, int64_t cap);
  * training run have close thresholds.  Results are identical either way (every bound is verified
  * by the exact count of the components it admits, and a row whose bound fails is redone exactly
  * in the same step); only the time differs: a step whose vectors differ a lot in scale from the
- * step before pays one multi-pass redo.  tk_set_bound_reuse(ctx, 0) samples every step.
+ * step before pays one multi-pass redo, after which its rows are sampled for 2, 4, ... up to 64
+ * steps before a bound is kept again.  tk_set_bound_reuse(ctx, 0) samples every step.
  */
 int tk_set_bound_reuse(tk_ctx* ctx, int on);
 

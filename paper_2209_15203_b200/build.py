@@ -33,15 +33,34 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
+def _deps():
+    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
+    deps.append(os.path.join(os.path.dirname(_HERE), "include", "topk.h"))
+    return deps
+
+
+def _compile(out: str, extra=(), verbose: bool = False) -> None:
+    tmp = out + ".tmp.%d" % os.getpid()
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
+           *[os.path.join(CSRC, s) for s in SOURCES]]
+    subprocess.run(cmd, check=True, cwd=CSRC)
+    os.replace(tmp, out)
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile the CUDA library if it is missing or older than its sources."""
     if force or _stale():
-        tmp = LIB + ".tmp.%d" % os.getpid()
-        cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
-               *[os.path.join(CSRC, s) for s in SOURCES]]
-        subprocess.run(cmd, check=True, cwd=CSRC)
-        os.replace(tmp, LIB)
+        _compile(LIB, verbose=verbose)
     return LIB
+
+
+def build_phase_clock(force: bool = False) -> str:
+    """The same library with the device phase clock compiled in (-DTK_PHASE_CLOCK=1), as
+    libtopk_clock.so beside the ordinary one; select it with TOPK_LIBRARY (see phase_clock.py)."""
+    out = os.path.join(_HERE, "libtopk_clock.so")
+    if force or not os.path.exists(out) or any(os.path.getmtime(p) > os.path.getmtime(out) for p in _deps()):
+        _compile(out, extra=["-DTK_PHASE_CLOCK=1"])
+    return out
 
 
 if __name__ == "__main__":

@@ -73,6 +73,7 @@ constexpr int kGridScratchWords = 3 * kHistBins + 4 + 2 * kRankMax;
 constexpr int kMaxRowsPerLaunch = 4096;
 constexpr u32 kRowGeneral = 1u;        // RowState.flags: row redone by the multi-pass path
 constexpr u32 kRowNoFilter = 2u;       // RowState.flags: no filter pass has read this row
+constexpr u32 kRowReused = 4u;         // RowState.flags: the row's bound was kept from its last selection, not sampled
 
 // Per-row state of one batched selection.  Lives in global memory.
 struct RowState {
@@ -94,7 +95,8 @@ struct RowState {
     u32 bin_base;    // union: a key no unshared sum of this step lies below (see union_base)
     u32 bin_hint;    // union: where the previous step's downlink threshold puts the buckets (0: none yet); survives resets
     u32 reuse_ok;    // the bound `lo` served the last selection well and may serve the next one (see predict_kernel); survives resets
-    u32 pad_;
+    u32 reuse_wait;  // bit 0..15: selections to sample before a bound may be kept again; bits 16..31: the current
+                     // back-off (doubles, up to 64, each time a kept bound fails; halves when one holds); survives resets
 };
 
 // Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the

@@ -48,6 +48,9 @@ namespace tk {
 // result stays exact either way — the bound is verified by the exact count as always, and a row
 // whose count leaves the window is sampled again in the step after (a row whose count falls
 // below K or above the list's capacity is redone by the multi-pass path in the same step).
+// A row whose kept bound failed is sampled for the next 2, 4, ... 64 selections before a bound
+// is kept again (rows whose threshold jumps from step to step — tie groups around the K-th
+// value — then cost one failed attempt in 64 steps instead of one in two).
 __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->lo = lo;
     r->cand_count = 0;
@@ -80,7 +83,7 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
     if (reuse && rs[row].reuse_ok) {  // the same answer in all CTAs of the row: nothing here writes reuse_ok
         if (t == 0) {
-            reset_state(rs + row, rs[row].lo, 0u);
+            reset_state(rs + row, rs[row].lo, kRowReused);
             phase_stamp(ctrl, kStampPredictEnd);
         }
         return;
@@ -1154,11 +1157,22 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         }
     }
     if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
-    // may the row's bound serve the next selection too?  (cand_count is not written by this kernel)
+    // may the row's bound serve the next selection too?  (cand_count and flags are not written by this kernel)
     if (!kGrid && !kDense && rank == 0 && threadIdx.x == 0) {
         const u64 cc = r->cand_count;
-        r->reuse_ok = ((r->flags & kRowGeneral) == 0u && (u32)r->lo == 0u && r->lo != 0ull && cc * 4u >= (u64)K * 5u &&
-                       cc <= (u64)K * 4u && cc <= (u64)cap) ? 1u : 0u;
+        const bool redone = (r->flags & kRowGeneral) != 0u, kept = (r->flags & kRowReused) != 0u;
+        u32 wait = r->reuse_wait & 0xffffu, backoff = r->reuse_wait >> 16;
+        if (kept && redone) {            // a kept bound failed: sample for a while, twice as long as last time
+            backoff = backoff < 2u ? 2u : (backoff < 64u ? backoff * 2u : 64u);
+            wait = backoff;
+        } else if (kept) {               // a kept bound held
+            backoff >>= 1;
+        }
+        bool ok = !redone && (u32)r->lo == 0u && r->lo != 0ull && cc * 4u >= (u64)K * 5u && cc <= (u64)K * 4u &&
+                  cc <= (u64)cap;
+        if (wait > 0u) { ok = false; --wait; }
+        r->reuse_ok = ok ? 1u : 0u;
+        r->reuse_wait = (backoff << 16) | wait;
     }
     // the next step's first level is centred on this step's threshold (every CTA is past its last look
     // at the buckets: a grid barrier lies behind whenever they were used)

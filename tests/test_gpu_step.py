@@ -152,9 +152,19 @@ def test_kept_bounds_survive_changes_of_scale():
             w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, 1, wl.K_down[0], "scale %g reuse=%s" % (c, reuse))
             general.append(ctx.tk_status().rows_general)
         if reuse:
-            assert general == [0, 0, wl.N, 0, 0, wl.N, 0, 0, 0], general
+            # (after a failed attempt the rows sample for two steps before a bound is kept again)
+            assert general == [0, 0, wl.N, 0, 0, 0, 0, 0, 0] or general == [0, 0, wl.N, 0, 0, wl.N, 0, 0, 0], general
         else:
             assert general == [0] * len(scales), general
+        if reuse:
+            # thresholds that jump every step: the back-off (2, 4, 8 ... steps of sampling after each failed
+            # attempt) keeps the failed attempts few
+            failed = 0
+            for s in range(14):
+                G = W.make_grads(wl, 20 + s, DEV) * (1e-3 if s % 2 else 1.0)
+                w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, 1, wl.K_down[0], "alternating scale step %d" % s)
+                failed += 1 if ctx.tk_status().rows_general else 0
+            assert failed <= 3, failed
         ctx.close()
 
 
