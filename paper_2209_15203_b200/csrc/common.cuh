@@ -27,10 +27,10 @@ constexpr int kPredictThreads = 1024;
 constexpr int kSampleSlots = kPredictCtas * kPredictThreads / 2;  // per-row sample maxima (one per thread pair)
 constexpr int kPredictMaxTurns = 10;   // 16-byte loads one sampling thread issues, all at once
 constexpr int kPredictLightTurns = 2;  // ... in the variant for many rows
-// Streaming passes.  Measured on B200: read bandwidth peaks with about 900-1150 threads and
-// 65-80 KB of loads in flight per SM and falls off sharply on either side (more resident
-// threads or deeper unrolling lose 20 %), so the filter kernel runs 2 CTAs of 448 threads
-// per SM with 5 x 16 bytes in flight per thread, as one wave.
+// Streaming passes.  Measured on B200 (448 threads x 2 CTAs per SM, one wave): read bandwidth
+// rises with the 16-byte loads a thread has in flight up to 8 (115 KB per SM: 5 -> 6 -> 8 loads take
+// 4 and 7 us off the 0.57 ms kernel of the benchmark workload), is no better at 10, and falls with
+// more resident threads (512 x 2) or fewer (320 .. 416 x 2 with 8 .. 10 loads).
 #ifndef TK_FILTER_THREADS
 #define TK_FILTER_THREADS 448
 #endif
@@ -43,8 +43,12 @@ constexpr int kPredictLightTurns = 2;  // ... in the variant for many rows
 constexpr int kFilterThreads = TK_FILTER_THREADS;  // filter kernel: threads per CTA
 constexpr int kFilterCtasPerSm = TK_FILTER_CTAS;   // filter kernel: resident CTAs per SM (grid = that x SMs)
 constexpr int kGeneralThreads = 512;               // multi-pass kernel: threads per CTA
-constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // 16-byte loads in flight per thread
-constexpr int kFilterTileVecs = kFilterThreads * kStreamUnroll;    // float4 per tile
+#ifndef TK_FILTER_UNROLL
+#define TK_FILTER_UNROLL 8
+#endif
+constexpr int kFilterUnroll = TK_FILTER_UNROLL;    // filter kernel: 16-byte loads in flight per thread
+constexpr int kStreamUnroll = TK_STREAM_UNROLL;    // multi-pass kernel: the same (512-thread CTAs; 8 measured 40 % slower there)
+constexpr int kFilterTileVecs = kFilterThreads * kFilterUnroll;    // float4 per tile
 constexpr int kGeneralTileVecs = kGeneralThreads * kStreamUnroll;
 #ifndef TK_FILTER_EF_UNROLL
 #define TK_FILTER_EF_UNROLL 2

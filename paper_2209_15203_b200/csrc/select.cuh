@@ -420,7 +420,7 @@ template <bool kEF, bool kStats>
 __global__ void __launch_bounds__(kFilterThreads, kFilterCtasPerSm)
 filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 parts, u32 cpp,
               RowState* rs, uint2* cand, u32 cap, EfArgs ef, Ctrl* ctrl) {
-    constexpr int kUnroll = kEF ? kFilterEfUnroll : kStreamUnroll;
+    constexpr int kUnroll = kEF ? kFilterEfUnroll : kFilterUnroll;
     extern __shared__ u64 sh_lo[];  // every row's bound, fetched once
     __shared__ uint2 sh_buf[(kFilterThreads / 32) * kStageSlots];
     __shared__ u32 sh_n[kFilterThreads / 32];
