@@ -798,7 +798,10 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     if (rc != TK_OK) return rc;
     // the downlink selection: the union can hold up to ucap entries, about 4096 per CTA, at most one
     // co-resident wave.  With more than one CTA its first level is counted by the server sum already.
-    int ctas = (int)((c->ucap + 4095) / 4096);
+#ifndef TK_DOWN_PER_CTA
+#define TK_DOWN_PER_CTA 4096
+#endif
+    int ctas = (int)((c->ucap + TK_DOWN_PER_CTA - 1) / TK_DOWN_PER_CTA);
     if (ctas > di->select_grid) ctas = di->select_grid;
     if (ctas < 1) ctas = 1;
     const bool prebuilt = bidir && !with_ef && ctas > 1;

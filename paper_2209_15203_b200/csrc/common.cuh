@@ -70,7 +70,10 @@ constexpr int kSelectThreads = 1024;   // cluster select: threads per CTA
 #define TK_SELECT_PER_THREAD 8
 #endif
 constexpr int kSelectPerThread = TK_SELECT_PER_THREAD;  // candidates per thread the cluster size aims at
-constexpr int kRankMax = 256;          // a bucket of at most this many candidates is ranked directly (cnt^2 compares) instead of refined
+#ifndef TK_RANK_MAX
+#define TK_RANK_MAX 256
+#endif
+constexpr int kRankMax = TK_RANK_MAX;          // a bucket of at most this many candidates is ranked directly (cnt^2 compares) instead of refined
 // Global scratch of the grid-wide select: three histograms, a counter (4 words) and a list of kRankMax
 // composite keys; all but the list must be zero when the kernel starts, and are when it ends.
 constexpr int kGridScratchWords = 3 * kHistBins + 4 + 2 * kRankMax;

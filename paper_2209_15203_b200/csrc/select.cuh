@@ -226,6 +226,9 @@ __device__ __forceinline__ RowGeom row_geom(const float* x, int row, int64_t d) 
 #ifndef TK_COOP_PDL
 #define TK_COOP_PDL 1
 #endif
+#ifndef TK_FILTER_DYN_MIN
+#define TK_FILTER_DYN_MIN 32
+#endif
 #ifndef TK_STAGE_SLOTS
 #define TK_STAGE_SLOTS 128
 #endif
@@ -443,11 +446,11 @@ filter_kernel(const float* __restrict__ x, int rows, int64_t d, u32 tpr, u32 par
     // their fixed shares a few per cent apart (measured on the benchmark workload: 545 .. 572 us,
     // no pattern from launch to launch), and with the claimed end they all run dry within a few
     // tiles' time of each other.
-    // (not for short ranges, under 64 tiles per CTA: there the barrier per claimed tile costs more than the
-    // fixed shares differ)
+    // (not for short ranges, under TK_FILTER_DYN_MIN = 32 tiles per CTA: there the barrier per claimed tile
+    // costs more than the fixed shares differ)
     u64 n_dyn = (u64)cpp * kFilterDynTiles;
     if (n_dyn > (t_end - t_begin) / 8) n_dyn = (t_end - t_begin) / 8;
-    if ((t_end - t_begin) < (u64)cpp * 64) n_dyn = 0;
+    if ((t_end - t_begin) < (u64)cpp * TK_FILTER_DYN_MIN) n_dyn = 0;
     const u64 t_dyn = t_end - n_dyn;
     u64 t = t_begin + (blockIdx.x - part * cpp);
     int cur = -1;
