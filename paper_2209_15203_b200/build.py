@@ -41,6 +41,8 @@ def _deps():
 
 def _compile(out: str, extra=(), verbose: bool = False) -> None:
     tmp = out + ".tmp.%d" % os.getpid()
+    # TOPK_NVCC_EXTRA: more flags, e.g. one of the tuning macros (-DTK_FILTER_DYN_TILES=0, -DTK_FILTER_UNROLL=5)
+    extra = [*extra, *os.environ.get("TOPK_NVCC_EXTRA", "").split()]
     cmd = [_nvcc(), *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
            *[os.path.join(CSRC, s) for s in SOURCES]]
     subprocess.run(cmd, check=True, cwd=CSRC)
