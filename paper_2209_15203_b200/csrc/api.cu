@@ -818,7 +818,7 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
         LinkArgs zero = {nullptr, nullptr, 0, 0, c->delta, (size_t)c->d, 0};
         ApplyArgs ap = {w_dev, 1.0f};
         rc = run_select(s, c->delta, 1, c->d, c->K_down, c->down, c->ctrl, c->force_general != 0, nullptr, nullptr,
-                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag);
+                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag, c->bound_reuse != 0);
         if (rc != TK_OK) return rc;
     } else if (bidir) {
         ApplyArgs ap = {w_dev, alpha};
