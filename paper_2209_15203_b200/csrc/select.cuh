@@ -2,10 +2,12 @@
 // steps of Algorithm 1/2) as four kernels:
 //
 //   predict_kernel   reads a small strided sample of every row and sets a
-//                    conservative lower bound `lo` on the K-th composite key
+//                    conservative lower bound `lo` on the K-th composite key — or
+//                    keeps the bound that served the row's last selection well
 //   filter_kernel    the one streaming pass over all rows*d values: appends every
 //                    component with ck >= lo to the row's candidate list and
-//                    counts them exactly
+//                    counts them exactly (tiles dealt out in advance, the last few
+//                    of each range claimed from a counter)
 //   general_kernel   verification + exact fallback.  A row whose count is below
 //                    K or above the list capacity (or every row, when no
 //                    prediction was made) gets its bound from full-row radix
