@@ -68,8 +68,12 @@ agg_link_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* 
 
 constexpr int kWindow = 128;  // consecutive workers whose terms one walk of a chain gathers (two 64-bit masks)
 
-// (256, 8): all 2048 threads of an SM stay resident — the kernel lives on memory parallelism
-__global__ void __launch_bounds__(256, 8)
+#ifndef TK_AGG_THREADS
+#define TK_AGG_THREADS 256
+#endif
+constexpr int kAggThreads = TK_AGG_THREADS;
+// all 2048 threads of an SM stay resident — the kernel lives on memory parallelism
+__global__ void __launch_bounds__(kAggThreads, 2048 / kAggThreads)
 agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float* __restrict__ p,
                   u32* head, u32* next, u32* slots, u32 row_words, RowState* uni /* the union's state */,
                   uint2* U, u32 ucap, float* w, float alpha, int apply, float* delta, Ctrl* ctrl, u32 d,

@@ -792,7 +792,7 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     // with memories the step size is already inside the messages
     const float scale = with_ef ? 1.0f : alpha;
     u32 total = (u32)(c->N * c->K_up);
-    u32 blocks = (total + 255) / 256;
+    u32 blocks = (total + kAggThreads - 1) / kAggThreads;
     DeviceInfo* di = nullptr;
     int rc = device_info(&di);
     if (rc != TK_OK) return rc;
@@ -805,7 +805,7 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
     if (ctas > di->select_grid) ctas = di->select_grid;
     if (ctas < 1) ctas = 1;
     const bool prebuilt = bidir && !with_ef && ctas > 1;
-    rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(256), 0, s, 0, (const uint2*)c->up.out, total,
+    rc = launch_dependent(agg_reduce_kernel, dim3(blocks), dim3(kAggThreads), 0, s, 0, (const uint2*)c->up.out, total,
                               (u32)c->K_up, (const float*)c->p, c->head, c->next, c->slots, c->slot_row_words, c->uni, c->U,
                               c->ucap, w_dev,
                               scale, bidir ? 0 : 1, (bidir && with_ef) ? c->delta : (float*)nullptr, c->ctrl, (u32)c->d,
