@@ -403,8 +403,9 @@ def main():
                     "parallelism": ("workers sharded over %d ranks, one all-gather per step" if args.sharded
                                     else "replicas x%d") % world,
                     "bounds": "sampled in every step" if args.no_bound_reuse else
-                              "kept from the step before where they admitted 1.25 K .. 4 K candidates (verified "
-                              "exactly every step), sampled otherwise; --no-bound-reuse samples every step"})
+                              "warm-started from the step before (last threshold minus a margin of 1.5-3 % or four times its "
+                              "recent movement; verified exactly every step), sampled otherwise; --no-bound-reuse samples "
+                              "every step"})
         if args.agree is not None:
             cfg["rows"] = "shared vector x (1 + %g z_q)" % args.agree
         cfg["input_checksum_step0"] = "%016x" % sum_checksum(bufs[0])

@@ -352,13 +352,16 @@ int tk_set_cand_cap(tk_ctx* ctx, int64_t cap);
  * Bound reuse (on by default; no counterpart in the paper, which says nothing about how Top_K is
  * computed).  The uplink selection of a long row first needs a lower bound of the row's K-th
  * magnitude; normally it is estimated from a sample of the row at the start of every step.  With
- * reuse on, a row whose bound admitted between 1.25 K and 4 K candidates in the context's last
- * step keeps that bound for the next step and skips the sampling — consecutive iterations of a
- * training run have close thresholds.  Results are identical either way (every bound is verified
+ * reuse on, a row starts from the threshold its selection found in the context's last step, minus
+ * a margin (1.5-3 % in value, four times the recent step-to-step movement of the row's threshold
+ * if that is more; rows whose threshold moves by more than 6-12 % a step are sampled), and skips
+ * the sampling — consecutive iterations of a training run have close thresholds.  Results are identical either way (every bound is verified
  * by the exact count of the components it admits, and a row whose bound fails is redone exactly
  * in the same step); only the time differs: a step whose vectors differ a lot in scale from the
- * step before pays one multi-pass redo, after which its rows are sampled for 2, 4, ... up to 64
- * steps before a bound is kept again.  tk_set_bound_reuse(ctx, 0) samples every step.
+ * step before pays one multi-pass redo, after which the context's rows are sampled for 2, 4, ...
+ * up to 1024 steps before warm starts are tried again.  Steps with the error memories (TK_MODE_EF)
+ * always sample: the compensated vectors pile up just under their thresholds, where a warm-started
+ * bound admits too much.  tk_set_bound_reuse(ctx, 0) samples every step.
  */
 int tk_set_bound_reuse(tk_ctx* ctx, int on);
 

@@ -85,6 +85,24 @@ agg_reduce_kernel(const uint2* __restrict__ up, u32 total, u32 K_up, const float
         for (int b = threadIdx.x; b < kHistBins; b += blockDim.x) sh_hist[b] = 0;
     dependency_wait();   // the entries are filed by the kernel before
     if (threadIdx.x == 0) phase_stamp(ctrl, kStampAggStart);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        // once per step: may the rows of the next step start from this step's thresholds?  Not for a
+        // while after a step in which a warm-started bound failed (2, 4, ... 1024 steps; see predict_kernel)
+        u32 wait = uni->reuse_wait & 0xffffu, backoff = uni->reuse_wait >> 16;
+        if (uni->reuse_fails) {
+            backoff = backoff < 2u ? 2u : (backoff < 1024u ? backoff * 2u : 1024u);
+            // an eighth of the rows or more at once is no accident: these vectors' thresholds do not hold still
+            if ((u64)uni->reuse_fails * 8u * K_up >= total && backoff < 64u) backoff = 64u;
+            wait = backoff;
+            uni->reuse_fails = 0;
+        } else if (uni->reuse_ok) {
+            backoff >>= 1;
+        }
+        const bool allow = wait == 0u;
+        if (wait) --wait;
+        uni->reuse_ok = allow ? 1u : 0u;
+        uni->reuse_wait = (backoff << 16) | wait;
+    }
     const u32 bin_base = level0 ? union_base(uni) : 0u;
     u32 e = blockIdx.x * blockDim.x + threadIdx.x;
     bool owner = false;

@@ -538,13 +538,13 @@ int run_select(cudaStream_t stream, const float* x, int64_t rows, int64_t d, int
             const bool light = turns <= (fused ? kPredictLightTurns / 2 : kPredictLightTurns);
             dim3 pg(kPredictCtas, nr);
             if (fused && light)
-                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
+                predict_kernel<true, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0, (const RowState*)link.uni);
             else if (fused)
-                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
+                predict_kernel<true, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0, (const RowState*)link.uni);
             else if (light)
-                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
+                predict_kernel<false, true><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0, (const RowState*)link.uni);
             else
-                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0);
+                predict_kernel<false, false><<<pg, kPredictThreads, 0, stream>>>(xb, d, turns, stride_fp, rank, (u32)K, rs, smax, ar, efb, ctrl, reuse ? 1 : 0, (const RowState*)link.uni);
             TK_LAUNCH_CHECK();
             if (ev0 && r0 == 0) cudaEventRecord(ev0, stream);
             u32 tprf = fused ? b.tpr_filter_ef : b.tpr_filter;
@@ -818,7 +818,7 @@ int run_server(tk_ctx* c, float* w_dev, float alpha, int mode) {
         LinkArgs zero = {nullptr, nullptr, 0, 0, c->delta, (size_t)c->d, 0};
         ApplyArgs ap = {w_dev, 1.0f};
         rc = run_select(s, c->delta, 1, c->d, c->K_down, c->down, c->ctrl, c->force_general != 0, nullptr, nullptr,
-                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag, c->bound_reuse != 0);
+                        &c->launches, nullptr, zero, EfArgs{nullptr, 0.0f}, ap, diag);
         if (rc != TK_OK) return rc;
     } else if (bidir) {
         ApplyArgs ap = {w_dev, alpha};
@@ -945,7 +945,7 @@ int enqueue_step(tk_ctx* c, float* w_dev, const float* grads_dev, float alpha, i
     SelectBufs up = c->up;
     if (c->cand_cap > 0) up.cap = capped(up.cap, c->cand_cap, c->K_up);  // shorter lists, packed closer in the same buffer
     rc = run_select(s, grads_dev, c->N, c->d, c->K_up, up, c->ctrl, c->force_general != 0, e0, e1,
-                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag, c->bound_reuse != 0);
+                    &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, diag, c->bound_reuse != 0 && !with_ef);
     if (rc != TK_OK) return rc;
     rc = run_server(c, w_dev, alpha, mode);
     if (rc != TK_OK || !gap) return rc;
@@ -979,12 +979,13 @@ int tk_step_uplink(tk_ctx* c, const float* grads_local_dev, int32_t row0, int32_
     b.cand += (size_t)row0 * b.cap;
     b.out += (size_t)row0 * (size_t)c->K_up;
     float* eps = with_ef ? c->eps + (size_t)row0 * (size_t)c->d : nullptr;
-    LinkArgs link = {nullptr, nullptr, 0, 0, eps, (size_t)c->d, 0};  // chains are built after the exchange
+    // (the entries are filed after the exchange; the union's state gates the rows' warm starts as in tk_step)
+    LinkArgs link = {nullptr, nullptr, 0, 0, eps, (size_t)c->d, 0, nullptr, 0, c->p, c->uni};
     EfArgs ef = {eps, alpha};
     // (the union's state is reset here too: the filing kernel of tk_step_server lowers its bin_base)
     return run_select(c->stream, grads_local_dev, rows, c->d, c->K_up, b, c->ctrl, c->force_general != 0, nullptr,
                       nullptr, &c->launches, c->uni, link, ef, ApplyArgs{nullptr, 0.0f}, c->diagnostics != 0,
-                      c->bound_reuse != 0);
+                      c->bound_reuse != 0 && !with_ef);
 }
 
 int tk_messages(tk_ctx* c, void** msgs_dev, size_t* bytes_per_row) {

@@ -101,9 +101,17 @@ struct RowState {
     u32 tile_ticket; // streaming pass: tiles handed out so far from the claimed end of tile range number <this row's index>
     u32 bin_base;    // union: a key no unshared sum of this step lies below (see union_base)
     u32 bin_hint;    // union: where the previous step's downlink threshold puts the buckets (0: none yet); survives resets
-    u32 reuse_ok;    // the bound `lo` served the last selection well and may serve the next one (see predict_kernel); survives resets
+    // warm start of the row's next selection (see predict_kernel); all of it survives resets
+    u32 reuse_ok;    // next_lo_key may serve as the next selection's bound
+    u32 next_lo_key; // the last threshold's key minus a margin
+    u32 prev_T_key;  // key of the K-th largest of the last selection (0: none)
+    u32 drift;       // how far, in keys, that key has recently moved from one selection to the next (decaying maximum)
     u32 reuse_wait;  // bit 0..15: selections to sample before a bound may be kept again; bits 16..31: the current
-                     // back-off (doubles, up to 64, each time a kept bound fails; halves when one holds); survives resets
+                     // back-off (doubles, up to 64, each time a warm-started bound fails; halves when one holds)
+    // In the union's state the three words above gate the warm starts of ALL rows of the context's next
+    // step (reuse_ok: allowed; reuse_wait: the same back-off, driven by reuse_fails), so that many rows
+    // with unsteady thresholds cannot each spend a failed attempt in turn.
+    u32 reuse_fails; // union: rows whose warm-started bound failed in this step
 };
 
 // Build with -DTK_PHASE_CLOCK=1 to make the kernels of a step leave device timestamps (the

@@ -43,16 +43,23 @@ namespace tk {
 // which costs two histogram passes instead of four — as the row's bound: at
 // least `rank` sampled values are >= it.
 //
-// Bound reuse.  Consecutive steps of a training run have close thresholds, so a bound that
-// admitted a comfortable number of candidates in the last selection of this row (between 1.25 K
-// and 4 K, all verified; RowState.reuse_ok, set by the selection kernel) is simply kept when
-// `reuse` is set: the row's CTAs return at once, no sample is read and nothing is ranked.  The
-// result stays exact either way — the bound is verified by the exact count as always, and a row
-// whose count leaves the window is sampled again in the step after (a row whose count falls
-// below K or above the list's capacity is redone by the multi-pass path in the same step).
-// A row whose kept bound failed is sampled for the next 2, 4, ... 64 selections before a bound
-// is kept again (rows whose threshold jumps from step to step — tie groups around the K-th
-// value — then cost one failed attempt in 64 steps instead of one in two).
+// Bound reuse.  Consecutive steps of a training run have close thresholds.  Every selection of
+// a row leaves the key of its K-th largest magnitude (prev_T_key) and a decaying maximum of how
+// far that key moved between consecutive selections (drift); the next selection's bound is that
+// key minus a margin of four times the drift — at least kReuseMinMargin keys, 1.5-3 % in value —
+// and with `reuse` set the row's CTAs return at once: no sample is read, nothing is ranked.  A
+// row whose threshold wanders gets a wider margin (more candidates); when four times the drift
+// exceeds kReuseMaxMargin (25-50 %) the row is sampled as usual.  The result stays exact either
+// way: the bound is verified by the exact count like a sampled one, and a row whose count falls
+// below K or above the list's capacity is redone by the multi-pass path in the same step, after
+// which it is sampled for the next 2, 4, ... 64 selections before a warm start is tried again.
+// Within a step of a context the back-off is shared by all rows (`gate`, the union's state,
+// updated once per step by the server sum): with many rows whose thresholds jump now and then
+// — tie groups around the K-th value — a failed attempt then costs one step in up to 1024,
+// not one row in every step.
+constexpr u32 kReuseMinMargin = 1u << 18;   // keys; a key step is 2^-23 .. 2^-24 of the value
+constexpr u32 kReuseMaxMargin = 1u << 22;
+constexpr u32 kReuseFirstDrift = 1u << 17;  // assumed before two thresholds have been seen
 __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
     r->lo = lo;
     r->cand_count = 0;
@@ -73,7 +80,8 @@ __device__ __forceinline__ void reset_state(RowState* r, u64 lo, u32 flags) {
 template <bool kEF, bool kLight>
 __global__ void __launch_bounds__(kPredictThreads, kLight ? 2 : 1)
 predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp, u32 rank, u32 K,
-               RowState* rs, u32* smax, RowState* also_reset, EfArgs ef, Ctrl* ctrl, int reuse) {
+               RowState* rs, u32* smax, RowState* also_reset, EfArgs ef, Ctrl* ctrl, int reuse,
+               const RowState* gate) {
     __shared__ u32 sh_hist[kHistBins];
     __shared__ u32 sh_scratch[33];
     __shared__ u32 sh_res[2];
@@ -83,9 +91,10 @@ predict_kernel(const float* __restrict__ x, int64_t d, int turns, u64 stride_fp,
     const int row = blockIdx.y;
     const u32 t = blockIdx.x * kPredictThreads + threadIdx.x;   // 0 .. 2*kSampleSlots-1
     if (also_reset && row == 0 && t == 0) reset_state(also_reset, 0ull, 0u);
-    if (reuse && rs[row].reuse_ok) {  // the same answer in all CTAs of the row: nothing here writes reuse_ok
+    // (the same answer in all CTAs of the row: nothing in this kernel writes either word)
+    if (reuse && rs[row].reuse_ok && (!gate || gate->reuse_ok)) {
         if (t == 0) {
-            reset_state(rs + row, rs[row].lo, kRowReused);
+            reset_state(rs + row, (u64)rs[row].next_lo_key << 32, kRowReused);
             phase_stamp(ctrl, kStampPredictEnd);
         }
         return;
@@ -1162,20 +1171,28 @@ select_kernel(const uint2* __restrict__ lists, size_t list_stride, u32 cap, RowS
         }
     }
     if (link.stats) warp_add_double(&r->sel_sq, sel_sq);
-    // may the row's bound serve the next selection too?  (cand_count and flags are not written by this kernel)
+    // warm start of the row's next selection (cand_count and flags are not written by this kernel)
     if (!kGrid && !kDense && rank == 0 && threadIdx.x == 0) {
-        const u64 cc = r->cand_count;
         const bool redone = (r->flags & kRowGeneral) != 0u, kept = (r->flags & kRowReused) != 0u;
+        const u32 Tkey = C > Keff ? (u32)(T >> 32) : 0u;  // 0: the whole list went out, there is no threshold
+        u32 drift = r->drift;
+        const u32 before = r->prev_T_key;
+        if (Tkey && before) drift = max(Tkey > before ? Tkey - before : before - Tkey, drift - drift / 16u);
+        else if (Tkey) drift = kReuseFirstDrift;
         u32 wait = r->reuse_wait & 0xffffu, backoff = r->reuse_wait >> 16;
-        if (kept && redone) {            // a kept bound failed: sample for a while, twice as long as last time
+        if (kept && redone) {            // a warm-started bound failed: sample for a while, twice as long as last time
             backoff = backoff < 2u ? 2u : (backoff < 64u ? backoff * 2u : 64u);
             wait = backoff;
-        } else if (kept) {               // a kept bound held
+            if (link.uni) atomicAdd(&link.uni->reuse_fails, 1u);  // ... and so do the context's other rows
+        } else if (kept) {               // a warm-started bound held
             backoff >>= 1;
         }
-        bool ok = !redone && (u32)r->lo == 0u && r->lo != 0ull && cc * 4u >= (u64)K * 5u && cc <= (u64)K * 4u &&
-                  cc <= (u64)cap;
+        const u64 margin = max((u64)kReuseMinMargin, 4ull * drift);
+        bool ok = !redone && (u32)r->lo == 0u && Tkey != 0u && margin <= (u64)kReuseMaxMargin && (u64)Tkey > margin;
         if (wait > 0u) { ok = false; --wait; }
+        r->prev_T_key = Tkey;
+        r->drift = drift;
+        r->next_lo_key = ok ? Tkey - (u32)margin : 0u;
         r->reuse_ok = ok ? 1u : 0u;
         r->reuse_wait = (backoff << 16) | wait;
     }

@@ -133,12 +133,12 @@ def test_forced_list_overflow_redoes_every_row_exactly():
 
 
 def test_kept_bounds_survive_changes_of_scale():
-    # A row keeps the bound of the step before when that bound admitted a comfortable number of
-    # candidates (tk_set_bound_reuse, on by default).  Steps of the same distribution then take the
-    # single streaming pass without sampling; a step whose vectors are a thousand times smaller (the
-    # kept bound admits nothing) or larger (it admits everything, the lists overflow) must be redone
-    # by the exact multi-pass path, and the step after that samples afresh.  Results are the oracle's
-    # throughout; with reuse off no step needs the multi-pass path.
+    # A row starts from the threshold of the step before, minus a margin (tk_set_bound_reuse, on by
+    # default).  Steps of the same distribution then take the single streaming pass without sampling; a
+    # step whose vectors are a thousand times smaller (the warm-started bound admits nothing) must be
+    # redone by the exact multi-pass path, and after such a jump the rows sample afresh (their
+    # thresholds have just shown that they move).  Results are the oracle's throughout; with reuse off
+    # no step needs the multi-pass path.
     wl = W.workload(2, d=700_003, N=5)
     scales = (1.0, 1.0, 1e-3, 1.0, 1.0, 1e3, 1.0, 0.97, 1.04)
     for reuse in (True, False):
@@ -183,6 +183,40 @@ def test_set_kdown_between_steps():
         ctx.tk_set_kdown(kd)
         G = W.make_grads(wl, s, DEV)
         w_ref = check_step(ctx, wl, w_dev, w_ref, G, 0.05, 1, kd, "set_kdown %d" % kd)
+
+
+def test_warm_started_steps_on_a_random_walk():
+    # What the library carries from step to step only steers speed: the rows' kept bounds and the
+    # centre of the downlink selection's first-level buckets.  Thirty steps whose scale drifts by up to
+    # +-15 % a step (sometimes jumping), with K_down and the mode changing under way, on a long-row
+    # workload whose union takes several CTAs: every step must equal the oracle's, with graph replay
+    # as the benchmark runs it.
+    rng = np.random.default_rng(2209)
+    for cid, d, N in ((2, 900_001, 12), (3, 600_002, 9)):
+        wl = W.workload(cid, d=d, N=N)
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            p = W.make_p(wl)
+            ctx = binding.Context(wl.d, wl.N, wl.K_up, wl.K_down[0], p, stream=stream)
+            _P[id(ctx)] = p.numpy()
+            ctx.tk_set_graph(True)
+            w_dev = W.make_w(wl, DEV)
+            w_ref = w_dev.cpu().numpy()
+            scale = 1.0
+            redone = 0
+            for s in range(30):
+                scale *= float(np.exp(rng.uniform(-0.15, 0.15)))
+                if s in (11, 23):
+                    scale *= 0.05 if s == 11 else 30.0
+                kd = int(rng.choice([wl.K_up, wl.K_up // 7 + 1, 5 * wl.K_up, wl.K_up]))
+                mode = int(rng.random() < 0.8)
+                ctx.tk_set_kdown(kd)
+                G = W.make_grads(wl, s, DEV) * scale
+                torch.cuda.synchronize()
+                w_ref = check_step(ctx, wl, w_dev, w_ref, G, wl.alpha, mode, kd, "walk config%d step %d scale %.3g" % (cid, s, scale))
+                redone += 1 if ctx.tk_status().rows_general else 0
+            assert redone <= 6, redone       # the two jumps, and what a 15 % drift occasionally costs
+            ctx.close()
 
 
 def test_cancelling_workers_and_zero_weights():
