@@ -254,6 +254,25 @@ def test_many_workers(N, d, K_up, K_down):
         ctx.close()
 
 
+@pytest.mark.parametrize("N,d,K_up", [(128, 400_003, 2500), (200, 300_002, 1600)])
+def test_more_entries_than_one_wave_of_server_threads(N, d, K_up):
+    # N*K_up above 148 * 2048 threads: the server sum runs in several waves of CTAs, with the slot table
+    # (N = 128) and with chains (N = 200); each coordinate is sent by 1.6 workers on average
+    rng = np.random.default_rng(N + K_up)
+    p = torch.from_numpy((rng.random(N) / N).astype(np.float32))
+    wl = W.workload(1, d=d, N=N)
+    K_down = 3 * K_up
+    wl = wl.__class__(**{**wl.__dict__, "K_up": K_up, "K_down": (K_down,)})
+    ctx = binding.Context(d, N, K_up, K_down, p)
+    _P[id(ctx)] = p.numpy()
+    w_dev = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+    w_ref = w_dev.cpu().numpy()
+    for s, mode in enumerate((1, 0, 1)):
+        G = torch.from_numpy(rng.standard_normal((N, d), dtype=np.float32)).to(DEV)
+        w_ref = check_step(ctx, wl, w_dev, w_ref, G, 0.05, mode, K_down, "N=%d K_up=%d mode=%d step=%d" % (N, K_up, mode, s))
+    ctx.close()
+
+
 @pytest.mark.parametrize("N,noise", [(20, 0.01), (100, 0.01), (150, 0.0)])
 def test_workers_that_agree(N, noise):
     # correlated gradients: almost every selected coordinate is sent by all N workers, so the sums
