@@ -30,3 +30,25 @@ def test_record_covers_every_configured_leg_without_a_mismatch():
                 assert idx_bad == 0 and not_equal == 0 and compared > 0, (key, rows[key])
                 want += 1
     assert len(rows) == want
+
+
+def test_record_with_error_memories_covers_the_four_large_workloads_without_a_mismatch():
+    """profiles/acceptance_error_memories.md: Algorithm 1 / 2 with the memories kept, configs 2-5 at full
+    size, every mode a config names; at least two consecutive steps (state carried), nothing differing."""
+    text = open(os.path.join(ROOT, "profiles", "acceptance_error_memories.md")).read()
+    rows = {}
+    for line in text.splitlines():
+        m = re.match(r"^\| (\d+) \| (unidirectional|bidirectional) \| (\d+) \| (\d+) \| (\d+) \| (\d+) \| (\d+) \|", line)
+        if m:
+            cid, mode, kdown, steps, idx_bad, compared, not_equal = m.groups()
+            rows[(int(cid), mode)] = (int(kdown), int(steps), int(idx_bad), int(compared), int(not_equal))
+    for cid in (2, 3, 4, 5):
+        wl = W.workload(cid)
+        for mode in wl.modes:
+            key = (cid, "bidirectional" if mode == 1 else "unidirectional")
+            assert key in rows, "no record of %r" % (key,)
+            kdown, steps, idx_bad, compared, not_equal = rows[key]
+            assert kdown == wl.K_down[0] and steps >= 2, (key, rows[key])
+            # the memories of all workers are among the values compared
+            assert compared >= steps * wl.N * wl.d, (key, rows[key])
+            assert idx_bad == 0 and not_equal == 0, (key, rows[key])
